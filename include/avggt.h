@@ -1,0 +1,164 @@
+/*
+ * avggt.h - C ABI of libavggt: subsampled global self-attention for
+ * VGGT / pi^3 style alternating frame/global transformers on NVIDIA B200
+ * (sm_100a).
+ *
+ * The library implements one layer of the AVGGT paper, "Subsampling Global
+ * Attention" (Sec. 4.3): every token of all N frames is a query; the keys and
+ * values are (i) all special tokens plus the first patch token of every
+ * s_h x s_w window of each frame's patch grid, (ii) the query's own key/value
+ * (diagonal preservation) and (iii) one mean key/value pair standing for all
+ * dropped patch tokens (mean-fill), normalised by one shared softmax.
+ *
+ * Conventions that hold for every entry point
+ *   - Plain C types only.  Pointers marked "device" are CUDA device pointers
+ *     on the current device; pointers marked "host" are ordinary host memory.
+ *   - The library never allocates or frees memory the caller can see.  All
+ *     buffers, including the workspace, are owned by the caller and must stay
+ *     valid until the work enqueued on the stream has finished.
+ *   - Device buffers must be 16-byte aligned (AVGGT_ERR_ALIGNMENT otherwise).
+ *   - Calls that take a stream only enqueue work on it and return without
+ *     synchronising.  `cuda_stream` is a cudaStream_t passed as void*
+ *     (NULL = the legacy default stream).
+ *   - Return value: 0 on success, a negative AVGGT_ERR_* code otherwise.
+ *     Arguments are validated on the host before anything is launched; on an
+ *     error nothing has been enqueued.  No exception crosses this boundary.
+ *   - Only sm_100 devices are supported (AVGGT_ERR_UNSUPPORTED elsewhere).
+ *     There is no CPU fallback.
+ *   - Calls on distinct streams with distinct output/workspace buffers may be
+ *     made from different host threads.
+ *
+ * Token layout (Sec. 4.1 notation): a frame has L = n_special + n_h*n_w
+ * tokens; slots [0, n_special) of a frame are its special tokens (camera and
+ * register tokens), followed by the patch grid in row-major order.  Token t
+ * of the sequence is slot t % L of frame t / L.  Q, K, V and O are
+ * [N*L, H, d] arrays, d contiguous, i.e. what a fused QKV projection
+ * produces for the (B, N*L, C) global layout of Sec. 4.2 with C = H*d.
+ */
+#ifndef AVGGT_H_
+#define AVGGT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AVGGT_OK                        0
+#define AVGGT_ERR_INVALID_ARG          -1   /* NULL pointer, non-positive size, inconsistent sizes   */
+#define AVGGT_ERR_UNSUPPORTED          -2   /* sigma, head_dim, batch, device not supported           */
+#define AVGGT_ERR_WORKSPACE_TOO_SMALL  -3
+#define AVGGT_ERR_ALIGNMENT            -4   /* a device pointer is not 16-byte aligned                */
+#define AVGGT_ERR_CUDA                 -5   /* a CUDA runtime/driver call failed; see avggt_last_cuda_error */
+#define AVGGT_ERR_DEVICE_TIMEOUT       -6   /* a bounded device-side wait ran out (avggt_check_status) */
+
+/* flags */
+#define AVGGT_FLAG_KEEP_FIRST_FRAME    1u   /* frame 0 keeps all patch K/V (VGGT variant, Sec. 4.3)   */
+
+/* mean_fill modes */
+#define AVGGT_MEAN_OFF     0
+#define AVGGT_MEAN_UNIT    1   /* the mean pair is one extra column of weight 1                       */
+#define AVGGT_MEAN_FILL    2   /* every dropped column is filled with the mean pair: the single mean  */
+                               /* column carries the count of columns it stands for                   */
+
+/*
+ * Problem statement (Sec. 4.1 and 4.3).  Plain data, passed by pointer (host).
+ */
+typedef struct avggt_params {
+  int32_t batch;             /* B; must be 1 (independent problems are separate calls)                */
+  int32_t n_frames;          /* N >= 1                                                                */
+  int32_t tokens_per_frame;  /* L; must equal n_special + grid_h * grid_w                             */
+  int32_t grid_h, grid_w;    /* n_h, n_w: patch grid of one frame                                     */
+  int32_t n_special;         /* special tokens per frame (5 for VGGT and pi^3), >= 0                  */
+  int32_t n_heads;           /* H >= 1                                                                */
+  int32_t head_dim;          /* d; must be 64                                                         */
+  int32_t sigma;             /* subsampling factor: 1 (dense), 2, 4, 6, 9 -> (s_h, s_w) =
+                                (1,1), (1,2), (2,2), (2,3), (3,3)  (Sec. 4.3, Subsampling Strategy)   */
+  int32_t diag;              /* 0/1: diagonal preservation                                            */
+  int32_t mean_fill;         /* AVGGT_MEAN_*                                                          */
+  float   softmax_scale;     /* <= 0 selects 1/sqrt(d)                                                */
+  uint32_t flags;            /* AVGGT_FLAG_*; unknown bits are rejected                               */
+} avggt_params;
+
+/*
+ * Number of compacted keys M and of dropped patch tokens |D| for a problem
+ * (Sec. 4.3: special tokens are always kept; a partial window at the grid
+ * edge keeps its first token).  Host-only, pure.
+ */
+int avggt_kv_count(const avggt_params* p, int64_t* n_kept, int64_t* n_dropped);
+
+/*
+ * Workspace sizes in bytes needed by avggt_build_kv and avggt_global_attn for
+ * this problem on the current device.  Either output may be NULL.
+ * Host-only apart from a device-property query.
+ */
+int avggt_workspace_bytes(const avggt_params* p, size_t* build_ws_bytes, size_t* attn_ws_bytes);
+
+/*
+ * K/V compaction and mean-fill reduction (Sec. 4.3, Subsampling Strategy and
+ * Enhanced Subsampling).  One pass over K and V:
+ *   Kc[h][m][:] = K[idx[m]][h][:],  Vc likewise      (bit copies)
+ *   kmean[h][:] = mean over dropped patch tokens j of K[j][h][:]   (fp32), vmean likewise
+ * where idx[m] is the global token index of the m-th retained key in ascending
+ * order.
+ *
+ *   K, V    device, bf16 [N*L, H, d]             read only
+ *   Kc, Vc  device, bf16 [H, M, d]  (head-major) written
+ *   idx     device, int32 [M], may be NULL       written
+ *   kmean, vmean  device, float [H, d]           written when mean_fill != 0 and |D| > 0
+ *                                                (zero-filled when |D| == 0); may be NULL when
+ *                                                mean_fill == 0
+ *   ws      device scratch of at least build_ws_bytes; holds per-block partial sums and is
+ *           fully rewritten by each call, so it needs no initialisation.  The reduction order is
+ *           fixed: results are identical from run to run.
+ */
+int avggt_build_kv(const avggt_params* p, const void* K, const void* V,
+                   void* Kc, void* Vc, int32_t* idx, float* kmean, float* vmean,
+                   void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Subsampled global attention (Sec. 4.3): for every query token i and head h
+ *   O[i][h][:] = ( sum_{m<M} e^{l_m} Vc[h][m] + [i in D, diag] e^{l_d} V[i][h] + [c_i>0, mean] e^{l_mu} vmean[h] ) / Z
+ * with l_m = scale q.Kc[h][m], l_d = scale q.K[i][h], l_mu = scale q.kmean[h] (+ ln c_i in
+ * AVGGT_MEAN_FILL mode), c_i = |D| - [i in D and diag], and Z the sum of the same exponentials
+ * (one shared softmax over the three disjoint components).  A query whose own column is
+ * retained has no separate diagonal term.  With |D| = 0 the result is dense softmax attention.
+ * Arithmetic: bf16 operands, fp32 accumulation and softmax, probabilities rounded to bf16 for
+ * the value product, output rounded to bf16 (nearest even).
+ *
+ *   Q             device, bf16 [N*L, H, d]
+ *   K, V          device, bf16 [N*L, H, d]; read only when diag != 0 (may be NULL otherwise)
+ *   Kc, Vc        device, bf16 [H, M, d] from avggt_build_kv
+ *   kmean, vmean  device, float [H, d]; read only when mean_fill != 0 and |D| > 0
+ *   O             device, bf16 [N*L, H, d]       written
+ *   lse           device, float [N*L, H] or NULL: natural-log normaliser ln(Z) + max-shift
+ *   ws            device scratch of at least attn_ws_bytes; the first 16 bytes are a status
+ *                 block that the call clears and that avggt_check_status reads.
+ */
+int avggt_global_attn(const avggt_params* p, const void* Q, const void* K, const void* V,
+                      const void* Kc, const void* Vc, const float* kmean, const float* vmean,
+                      void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * After the caller has synchronised the stream: reads the status block at the start of an
+ * attention workspace (a 16-byte device-to-host copy) and returns AVGGT_OK or
+ * AVGGT_ERR_DEVICE_TIMEOUT if a bounded wait inside the kernel gave up (the output is then
+ * undefined; the context stays usable).  `detail`, if not NULL, receives the raw status words
+ * (host, 4 x uint32: code, block, role/stage, iteration).
+ */
+int avggt_check_status(const void* attn_ws, uint32_t* detail);
+
+/* Static description of an error code. */
+const char* avggt_strerror(int code);
+
+/* Text of the last CUDA error seen by this thread inside the library ("" if none). */
+const char* avggt_last_cuda_error(void);
+
+/* Library version, "major.minor.patch". */
+const char* avggt_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AVGGT_H_ */

@@ -139,32 +139,35 @@ def kv_count(cfg):
 def build_kv(cfg, K, V):
     """Gather K_S, V_S and the mean pair over D.
 
-    K, V: arrays [N*L, H, d] (any real dtype; widened to float64).
+    K, V: arrays [N*L, H, d] (any real dtype; every value that is used is
+    widened to float64 before any arithmetic).
     Returns (Kc [M,H,d], Vc [M,H,d], idx [M] int32, kmean [H,d], vmean [H,d]).
     kmean/vmean are None when D is empty.
     """
-    K = np.asarray(K, dtype=np.float64)
-    V = np.asarray(V, dtype=np.float64)
+    K = np.asarray(K)
+    V = np.asarray(V)
     assert K.shape == (cfg.n_tokens, cfg.n_heads, cfg.head_dim) and V.shape == K.shape
     idx = build_index(cfg)
     dropped = dropped_token_mask(cfg)
-    Kc = K[idx]
-    Vc = V[idx]
+    Kc = K[idx].astype(np.float64)
+    Vc = V[idx].astype(np.float64)
     if dropped.any():
-        kmean = K[dropped].mean(axis=0)
-        vmean = V[dropped].mean(axis=0)
+        kmean = K[dropped].mean(axis=0, dtype=np.float64)
+        vmean = V[dropped].mean(axis=0, dtype=np.float64)
     else:
         kmean = vmean = None
     return Kc, Vc, idx, kmean, vmean
 
 
-def global_attn(cfg, Q, K, V, rows=None, return_weights=False):
+def global_attn(cfg, Q, K, V, rows=None, return_weights=False, return_lse=False):
     """Subsampled global attention for the query rows ``rows`` (default: all).
 
     Q, K, V: [N*L, H, d].  Returns O [len(rows), H, d] float64, and with
     ``return_weights`` also a list (one entry per row) of dicts with the
     softmax weights of the three components per head:
-    {'subset': [H, M], 'diag': [H] or None, 'mean': [H] or None}.
+    {'subset': [H, M], 'diag': [H] or None, 'mean': [H] or None}; with
+    ``return_lse`` also the natural-log normaliser ln(sum of exponentials of
+    all present logits) as [len(rows), H].
     """
     Q = np.asarray(Q, dtype=np.float64)
     K = np.asarray(K, dtype=np.float64)
@@ -184,6 +187,7 @@ def global_attn(cfg, Q, K, V, rows=None, return_weights=False):
         rows = np.arange(cfg.n_tokens)
     rows = np.asarray(rows, dtype=np.int64)
     O = np.empty((len(rows), H, d), dtype=np.float64)
+    lse = np.empty((len(rows), H), dtype=np.float64)
     weights = [] if return_weights else None
 
     for out_i, i in enumerate(rows):
@@ -207,9 +211,11 @@ def global_attn(cfg, Q, K, V, rows=None, return_weights=False):
             parts.append(logit_m[:, None])
         logits = np.concatenate(parts, axis=1)          # [H, M (+1) (+1)]
         # one shared softmax normalisation over all components
-        logits = logits - logits.max(axis=1, keepdims=True)
-        p = np.exp(logits)
-        p /= p.sum(axis=1, keepdims=True)
+        mx = logits.max(axis=1, keepdims=True)
+        p = np.exp(logits - mx)
+        z = p.sum(axis=1, keepdims=True)
+        p /= z
+        lse[out_i] = (mx + np.log(z))[:, 0]
         M = logit_s.shape[1]
         o = np.einsum("hm,hmd->hd", p[:, :M], Vc_h)
         col = M
@@ -224,36 +230,41 @@ def global_attn(cfg, Q, K, V, rows=None, return_weights=False):
         O[out_i] = o
         if return_weights:
             weights.append(w)
+    out = (O,)
     if return_weights:
-        return O, weights
-    return O
+        out += (weights,)
+    if return_lse:
+        out += (lse,)
+    return out[0] if len(out) == 1 else out
 
 
-def global_attn_blocked(cfg, Q, K, V, rows):
+def global_attn_blocked(cfg, Q, K, V, rows, return_lse=False):
     """Same result as ``global_attn`` for many rows at once (one matmul per
     head over all requested rows instead of one per row).  Used where the
     per-row loop would take minutes; checked against ``global_attn`` in the
     tests.  The arithmetic per row is unchanged.
     """
-    Q = np.asarray(Q, dtype=np.float64)
-    K = np.asarray(K, dtype=np.float64)
-    V = np.asarray(V, dtype=np.float64)
+    Q, K, V = np.asarray(Q), np.asarray(K), np.asarray(V)
     H, d = cfg.n_heads, cfg.head_dim
     scale = cfg.scale
     rows = np.asarray(rows, dtype=np.int64)
     Kc, Vc, idx, kmean, vmean = build_kv(cfg, K, V)
+    Q_r = Q[rows].astype(np.float64)      # only the requested rows are widened
+    K_r = K[rows].astype(np.float64)
+    V_r = V[rows].astype(np.float64)
     dropped = dropped_token_mask(cfg)
     n_dropped = int(dropped.sum())
     O = np.empty((len(rows), H, d), dtype=np.float64)
+    lse = np.empty((len(rows), H), dtype=np.float64)
     row_dropped = dropped[rows]
     has_diag = row_dropped & bool(cfg.diag)
     count = n_dropped - has_diag.astype(np.int64)
     has_mean = (count > 0) & (cfg.mean_fill != 0)
     NEG = -np.inf
     for h in range(H):
-        q = Q[rows, h, :]                                # [R, d]
+        q = Q_r[:, h, :]                                 # [R, d]
         logit_s = scale * (q @ Kc[:, h, :].T)            # [R, M]
-        logit_d = np.where(has_diag, scale * np.sum(q * K[rows, h, :], axis=1), NEG)
+        logit_d = np.where(has_diag, scale * np.sum(q * K_r[:, h, :], axis=1), NEG)
         if kmean is not None:
             lm = scale * (q @ kmean[h])
             if cfg.mean_fill == 2:
@@ -267,8 +278,9 @@ def global_attn_blocked(cfg, Q, K, V, rows):
         p_m = np.exp(logit_m - mx)
         z = p_s.sum(axis=1) + p_d + p_m
         o = p_s @ Vc[:, h, :]
-        o += p_d[:, None] * V[rows, h, :]
+        o += p_d[:, None] * V_r[:, h, :]
         if kmean is not None:
             o += p_m[:, None] * vmean[h][None, :]
         O[:, h, :] = o / z[:, None]
-    return O
+        lse[:, h] = mx + np.log(z)
+    return (O, lse) if return_lse else O

@@ -1,0 +1,8 @@
+"""B200-native subsampled global attention (AVGGT, Sec. 4.3): Python binding of libavggt."""
+
+from .binding import (  # noqa: F401
+    AVGGT_FLAG_KEEP_FIRST_FRAME, AVGGT_MEAN_FILL, AVGGT_MEAN_OFF, AVGGT_MEAN_UNIT, AvggtError, AvggtParams,
+    avggt_build_kv, avggt_check_status, avggt_global_attn, avggt_kv_count, avggt_version, avggt_workspace_bytes,
+    make_params,
+)
+from .layer import SubsampledGlobalAttention  # noqa: F401

@@ -1,0 +1,150 @@
+"""ctypes binding of libavggt.so: same names as the C ABI, argument marshalling only.
+
+Every step of the path runs inside the library's CUDA kernels.  There is no
+fallback: if the shared library is missing and cannot be built, importing the
+entry points raises.
+"""
+
+import ctypes
+import os
+
+from . import build as _build
+
+AVGGT_OK = 0
+AVGGT_ERR_INVALID_ARG = -1
+AVGGT_ERR_UNSUPPORTED = -2
+AVGGT_ERR_WORKSPACE_TOO_SMALL = -3
+AVGGT_ERR_ALIGNMENT = -4
+AVGGT_ERR_CUDA = -5
+AVGGT_ERR_DEVICE_TIMEOUT = -6
+
+AVGGT_FLAG_KEEP_FIRST_FRAME = 1
+AVGGT_MEAN_OFF, AVGGT_MEAN_UNIT, AVGGT_MEAN_FILL = 0, 1, 2
+
+# every symbol include/avggt.h declares
+EXPORTS = (
+    "avggt_kv_count", "avggt_workspace_bytes", "avggt_build_kv", "avggt_global_attn",
+    "avggt_check_status", "avggt_strerror", "avggt_last_cuda_error", "avggt_version",
+)
+
+
+class AvggtParams(ctypes.Structure):
+    """Mirror of ``avggt_params`` in include/avggt.h."""
+
+    _fields_ = [
+        ("batch", ctypes.c_int32),
+        ("n_frames", ctypes.c_int32),
+        ("tokens_per_frame", ctypes.c_int32),
+        ("grid_h", ctypes.c_int32),
+        ("grid_w", ctypes.c_int32),
+        ("n_special", ctypes.c_int32),
+        ("n_heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32),
+        ("sigma", ctypes.c_int32),
+        ("diag", ctypes.c_int32),
+        ("mean_fill", ctypes.c_int32),
+        ("softmax_scale", ctypes.c_float),
+        ("flags", ctypes.c_uint32),
+    ]
+
+
+class AvggtError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        msg = lib().avggt_strerror(code).decode()
+        if code == AVGGT_ERR_CUDA:
+            msg += ": " + lib().avggt_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg} ({code})")
+
+
+_LIB = None
+
+
+def lib():
+    """The loaded shared library (built in-tree on first use if stale or absent)."""
+    global _LIB
+    if _LIB is None:
+        path = _build.LIB
+        if _build.needs_build():
+            try:
+                path = _build.build()
+            except Exception:
+                if not os.path.exists(_build.LIB):
+                    raise
+                path = _build.LIB      # no compiler on this machine: use the library that shipped
+        L = ctypes.CDLL(path)
+        vp, i64p, szp = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_size_t)
+        pp = ctypes.POINTER(AvggtParams)
+        L.avggt_kv_count.argtypes = [pp, i64p, i64p]
+        L.avggt_workspace_bytes.argtypes = [pp, szp, szp]
+        L.avggt_build_kv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.avggt_global_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.avggt_check_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+        L.avggt_strerror.argtypes = [ctypes.c_int]
+        for f in (L.avggt_kv_count, L.avggt_workspace_bytes, L.avggt_build_kv, L.avggt_global_attn, L.avggt_check_status):
+            f.restype = ctypes.c_int
+        for f in (L.avggt_strerror, L.avggt_last_cuda_error, L.avggt_version):
+            f.restype = ctypes.c_char_p
+        _LIB = L
+    return _LIB
+
+
+def make_params(n_frames, grid_h, grid_w, n_special, n_heads, head_dim, sigma, diag=1, mean_fill=AVGGT_MEAN_FILL,
+                softmax_scale=0.0, keep_first_frame=False, batch=1):
+    return AvggtParams(batch, n_frames, n_special + grid_h * grid_w, grid_h, grid_w, n_special, n_heads, head_dim,
+                       sigma, int(diag), int(mean_fill), float(softmax_scale),
+                       AVGGT_FLAG_KEEP_FIRST_FRAME if keep_first_frame else 0)
+
+
+def _check(code, where):
+    if code != AVGGT_OK:
+        raise AvggtError(code, where)
+
+
+def _ptr(t):
+    """Device (or host) address of a tensor-like object, or None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def avggt_kv_count(params):
+    """-> (M, n_dropped)."""
+    m, nd = ctypes.c_int64(), ctypes.c_int64()
+    _check(lib().avggt_kv_count(ctypes.byref(params), ctypes.byref(m), ctypes.byref(nd)), "avggt_kv_count")
+    return m.value, nd.value
+
+
+def avggt_workspace_bytes(params):
+    """-> (build_ws_bytes, attn_ws_bytes) on the current CUDA device."""
+    b, a = ctypes.c_size_t(), ctypes.c_size_t()
+    _check(lib().avggt_workspace_bytes(ctypes.byref(params), ctypes.byref(b), ctypes.byref(a)), "avggt_workspace_bytes")
+    return b.value, a.value
+
+
+def avggt_build_kv(params, K, V, Kc, Vc, idx, kmean, vmean, ws, ws_bytes, stream=None):
+    """Enqueue the K/V compaction + mean reduction.  Arguments are tensors (or raw addresses)."""
+    _check(lib().avggt_build_kv(ctypes.byref(params), _ptr(K), _ptr(V), _ptr(Kc), _ptr(Vc), _ptr(idx), _ptr(kmean),
+                                _ptr(vmean), _ptr(ws), ws_bytes, stream), "avggt_build_kv")
+
+
+def avggt_global_attn(params, Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws, ws_bytes, stream=None):
+    """Enqueue the subsampled global attention."""
+    _check(lib().avggt_global_attn(ctypes.byref(params), _ptr(Q), _ptr(K), _ptr(V), _ptr(Kc), _ptr(Vc), _ptr(kmean),
+                                   _ptr(vmean), _ptr(O), _ptr(lse), _ptr(ws), ws_bytes, stream), "avggt_global_attn")
+
+
+def avggt_check_status(attn_ws):
+    """After a stream synchronise: raises AvggtError if a device-side wait gave up."""
+    detail = (ctypes.c_uint32 * 4)()
+    code = lib().avggt_check_status(_ptr(attn_ws), detail)
+    if code != AVGGT_OK:
+        err = AvggtError(code, "avggt_check_status")
+        err.detail = tuple(detail)
+        raise err
+
+
+def avggt_version():
+    return lib().avggt_version().decode()

@@ -1,0 +1,198 @@
+// C ABI of libavggt: argument validation, the problem plan, and the launchers'
+// entry points.  Nothing here touches the data; every step of the path runs in
+// the kernels of build_kv.cu and global_attn.cu.
+#include <cmath>
+#include <cstring>
+#include <mutex>
+
+#include "internal.h"
+
+namespace avggt {
+
+namespace {
+
+thread_local char g_cuda_error[256] = "";
+
+int record_cuda(cudaError_t e) {
+  if (e == cudaSuccess) return AVGGT_OK;
+  std::strncpy(g_cuda_error, cudaGetErrorString(e), sizeof(g_cuda_error) - 1);
+  g_cuda_error[sizeof(g_cuda_error) - 1] = 0;
+  (void)cudaGetLastError();   // clear the sticky-less error state
+  return AVGGT_ERR_CUDA;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct DeviceInfo { int sm_count; int cc_major; };
+
+// Properties of the current device (queried once per device index).
+int device_info(DeviceInfo* out) {
+  static std::mutex mu;
+  static DeviceInfo cache[64];
+  static bool have[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return record_cuda(e);
+  std::lock_guard<std::mutex> lock(mu);
+  if (dev < 0 || dev >= 64) return AVGGT_ERR_UNSUPPORTED;
+  if (!have[dev]) {
+    DeviceInfo di;
+    e = cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return record_cuda(e);
+    e = cudaDeviceGetAttribute(&di.cc_major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return record_cuda(e);
+    cache[dev] = di;
+    have[dev] = true;
+  }
+  *out = cache[dev];
+  return out->cc_major == 10 ? AVGGT_OK : AVGGT_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+int make_plan(const avggt_params* p, Plan* pl) {
+  if (p == nullptr || pl == nullptr) return AVGGT_ERR_INVALID_ARG;
+  if (p->n_frames < 1 || p->grid_h < 1 || p->grid_w < 1 || p->n_special < 0 || p->n_heads < 1 || p->head_dim < 1)
+    return AVGGT_ERR_INVALID_ARG;
+  if (p->diag != 0 && p->diag != 1) return AVGGT_ERR_INVALID_ARG;
+  if (p->mean_fill < AVGGT_MEAN_OFF || p->mean_fill > AVGGT_MEAN_FILL) return AVGGT_ERR_INVALID_ARG;
+  if (p->flags & ~AVGGT_FLAG_KEEP_FIRST_FRAME) return AVGGT_ERR_INVALID_ARG;
+  if (!(p->softmax_scale == p->softmax_scale) || std::isinf(p->softmax_scale)) return AVGGT_ERR_INVALID_ARG;
+  const int64_t patches = static_cast<int64_t>(p->grid_h) * p->grid_w;
+  if (patches + p->n_special != p->tokens_per_frame) return AVGGT_ERR_INVALID_ARG;
+  if (p->batch != 1) return AVGGT_ERR_UNSUPPORTED;
+  if (p->head_dim != 64) return AVGGT_ERR_UNSUPPORTED;
+  if (p->n_heads > 32) return AVGGT_ERR_UNSUPPORTED;
+  int s_h, s_w;
+  switch (p->sigma) {   // Sec. 4.3, Subsampling Strategy
+    case 1: s_h = 1; s_w = 1; break;
+    case 2: s_h = 1; s_w = 2; break;
+    case 4: s_h = 2; s_w = 2; break;
+    case 6: s_h = 2; s_w = 3; break;
+    case 9: s_h = 3; s_w = 3; break;
+    default: return AVGGT_ERR_UNSUPPORTED;
+  }
+  const int64_t n_tok = static_cast<int64_t>(p->n_frames) * p->tokens_per_frame;
+  if (n_tok > 0x7fffffffll - 256) return AVGGT_ERR_UNSUPPORTED;
+  pl->n_frames = p->n_frames;
+  pl->L = p->tokens_per_frame;
+  pl->grid_h = p->grid_h;
+  pl->grid_w = p->grid_w;
+  pl->n_special = p->n_special;
+  pl->H = p->n_heads;
+  pl->d = p->head_dim;
+  pl->s_h = s_h;
+  pl->s_w = s_w;
+  pl->kept_w = (p->grid_w + s_w - 1) / s_w;
+  pl->kept_patches = ((p->grid_h + s_h - 1) / s_h) * pl->kept_w;
+  pl->Lc = p->n_special + pl->kept_patches;
+  pl->keep_first = (p->flags & AVGGT_FLAG_KEEP_FIRST_FRAME) ? 1 : 0;
+  pl->diag = p->diag;
+  pl->mean_fill = p->mean_fill;
+  pl->n_tok = n_tok;
+  pl->M = static_cast<int64_t>(p->n_frames) * pl->Lc + (pl->keep_first ? (patches - pl->kept_patches) : 0);
+  pl->n_dropped = n_tok - pl->M;
+  pl->scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / std::sqrt(static_cast<float>(p->head_dim));
+  if (pl->M < 1) return AVGGT_ERR_INVALID_ARG;
+  return AVGGT_OK;
+}
+
+}  // namespace avggt
+
+using namespace avggt;
+
+extern "C" {
+
+int avggt_kv_count(const avggt_params* p, int64_t* n_kept, int64_t* n_dropped) {
+  Plan pl;
+  int rc = make_plan(p, &pl);
+  if (rc != AVGGT_OK) return rc;
+  if (n_kept) *n_kept = pl.M;
+  if (n_dropped) *n_dropped = pl.n_dropped;
+  return AVGGT_OK;
+}
+
+int avggt_workspace_bytes(const avggt_params* p, size_t* build_ws_bytes, size_t* attn_ws_bytes) {
+  Plan pl;
+  int rc = make_plan(p, &pl);
+  if (rc != AVGGT_OK) return rc;
+  DeviceInfo di;
+  rc = device_info(&di);
+  if (rc != AVGGT_OK) return rc;
+  if (build_ws_bytes) *build_ws_bytes = build_kv_ws_bytes(pl, di.sm_count);
+  if (attn_ws_bytes) *attn_ws_bytes = global_attn_ws_bytes(pl, di.sm_count);
+  return AVGGT_OK;
+}
+
+int avggt_build_kv(const avggt_params* p, const void* K, const void* V, void* Kc, void* Vc, int32_t* idx,
+                   float* kmean, float* vmean, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Plan pl;
+  int rc = make_plan(p, &pl);
+  if (rc != AVGGT_OK) return rc;
+  if (!K || !V || !Kc || !Vc || !ws) return AVGGT_ERR_INVALID_ARG;
+  if (pl.mean_fill != 0 && (!kmean || !vmean)) return AVGGT_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(V) || !aligned16(Kc) || !aligned16(Vc) || !aligned16(ws) ||
+      (reinterpret_cast<uintptr_t>(idx) & 3u) || !aligned16(kmean) || !aligned16(vmean))
+    return AVGGT_ERR_ALIGNMENT;
+  DeviceInfo di;
+  rc = device_info(&di);
+  if (rc != AVGGT_OK) return rc;
+  if (ws_bytes < build_kv_ws_bytes(pl, di.sm_count)) return AVGGT_ERR_WORKSPACE_TOO_SMALL;
+  return record_cuda(launch_build_kv(pl, di.sm_count, K, V, Kc, Vc, idx, kmean, vmean, ws, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int avggt_global_attn(const avggt_params* p, const void* Q, const void* K, const void* V, const void* Kc,
+                      const void* Vc, const float* kmean, const float* vmean, void* O, float* lse, void* ws,
+                      size_t ws_bytes, void* cuda_stream) {
+  Plan pl;
+  int rc = make_plan(p, &pl);
+  if (rc != AVGGT_OK) return rc;
+  const bool need_diag = pl.diag != 0 && pl.n_dropped > 0;
+  const bool need_mean = pl.mean_fill != 0 && pl.n_dropped > 0;
+  if (!Q || !Kc || !Vc || !O || !ws) return AVGGT_ERR_INVALID_ARG;
+  if (need_diag && (!K || !V)) return AVGGT_ERR_INVALID_ARG;
+  if (need_mean && (!kmean || !vmean)) return AVGGT_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(Kc) || !aligned16(Vc) || !aligned16(O) ||
+      !aligned16(ws) || !aligned16(kmean) || !aligned16(vmean) || (reinterpret_cast<uintptr_t>(lse) & 3u))
+    return AVGGT_ERR_ALIGNMENT;
+  DeviceInfo di;
+  rc = device_info(&di);
+  if (rc != AVGGT_OK) return rc;
+  if (ws_bytes < global_attn_ws_bytes(pl, di.sm_count)) return AVGGT_ERR_WORKSPACE_TOO_SMALL;
+  bool tmap_failed = false;
+  cudaError_t e = launch_global_attn(pl, di.sm_count, Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws,
+                                     static_cast<cudaStream_t>(cuda_stream), &tmap_failed);
+  if (tmap_failed) {
+    std::strncpy(g_cuda_error, "cuTensorMapEncodeTiled failed", sizeof(g_cuda_error) - 1);
+    return AVGGT_ERR_CUDA;
+  }
+  return record_cuda(e);
+}
+
+int avggt_check_status(const void* attn_ws, uint32_t* detail) {
+  if (!attn_ws) return AVGGT_ERR_INVALID_ARG;
+  uint32_t st[4] = {0, 0, 0, 0};
+  cudaError_t e = cudaMemcpy(st, attn_ws, sizeof(st), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return record_cuda(e);
+  if (detail) std::memcpy(detail, st, sizeof(st));
+  return st[0] == 0 ? AVGGT_OK : AVGGT_ERR_DEVICE_TIMEOUT;
+}
+
+const char* avggt_strerror(int code) {
+  switch (code) {
+    case AVGGT_OK: return "success";
+    case AVGGT_ERR_INVALID_ARG: return "invalid argument";
+    case AVGGT_ERR_UNSUPPORTED: return "unsupported configuration or device";
+    case AVGGT_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case AVGGT_ERR_ALIGNMENT: return "device pointer not 16-byte aligned";
+    case AVGGT_ERR_CUDA: return "CUDA call failed";
+    case AVGGT_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+    default: return "unknown error code";
+  }
+}
+
+const char* avggt_last_cuda_error(void) { return g_cuda_error; }
+
+const char* avggt_version(void) { return "0.1.0"; }
+
+}  // extern "C"

@@ -299,5 +299,27 @@ def test_blocked_equals_rowwise(sigma, diag, mean_fill):
     cfg = orc.SGAConfig(3, 7, 6, 5, 3, 16, sigma=sigma, diag=diag, mean_fill=mean_fill)
     Q, K, V = _rand_qkv(cfg, seed=31)
     rows = np.arange(0, cfg.n_tokens, 3)
-    np.testing.assert_allclose(orc.global_attn_blocked(cfg, Q, K, V, rows),
-                               orc.global_attn(cfg, Q, K, V, rows=rows), rtol=0, atol=1e-12)
+    O_b, lse_b = orc.global_attn_blocked(cfg, Q, K, V, rows, return_lse=True)
+    O_r, lse_r = orc.global_attn(cfg, Q, K, V, rows=rows, return_lse=True)
+    np.testing.assert_allclose(O_b, O_r, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(lse_b, lse_r, rtol=0, atol=1e-12)
+    # float32 inputs (how bf16 tensors reach the oracle) are widened, not computed in
+    np.testing.assert_allclose(
+        orc.global_attn_blocked(cfg, Q.astype(np.float32), K.astype(np.float32), V.astype(np.float32), rows),
+        orc.global_attn(cfg, Q.astype(np.float32).astype(np.float64), K.astype(np.float32).astype(np.float64),
+                        V.astype(np.float32).astype(np.float64), rows=rows), rtol=0, atol=1e-12)
+
+
+def test_lse_is_log_of_summed_exponentials():
+    """The normaliser against a direct enumeration of the present columns."""
+    cfg = _tiny(4, True, 2)
+    Q, K, V = _rand_qkv(cfg, seed=37)
+    _, lse = orc.global_attn(cfg, Q, K, V, return_lse=True)
+    D = _dropped_by_slicing(cfg)
+    scale = 1.0 / math.sqrt(cfg.head_dim)
+    for i in (0, 3, 9, cfg.n_tokens - 1):
+        for h in range(cfg.n_heads):
+            kbar = K[D, h].mean(axis=0)
+            tot = sum(math.exp(scale * float(Q[i, h] @ K[j, h])) for j in range(cfg.n_tokens) if not D[j] or j == i)
+            tot += (int(D.sum()) - int(D[i])) * math.exp(scale * float(Q[i, h] @ kbar))
+            assert abs(lse[i, h] - math.log(tot)) < 1e-12
