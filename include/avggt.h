@@ -52,6 +52,7 @@ extern "C" {
 #define AVGGT_ERR_ALIGNMENT            -4   /* a device pointer is not 16-byte aligned                */
 #define AVGGT_ERR_CUDA                 -5   /* a CUDA runtime/driver call failed; see avggt_last_cuda_error */
 #define AVGGT_ERR_DEVICE_TIMEOUT       -6   /* a bounded device-side wait ran out (avggt_check_status) */
+#define AVGGT_ERR_STATIC_SCRATCH       -7   /* problem exceeds the fixed scratch of avggt_build_kv_noalloc */
 
 /* flags */
 #define AVGGT_FLAG_KEEP_FIRST_FRAME    1u   /* frame 0 keeps all patch K/V (VGGT variant, Sec. 4.3)   */
@@ -116,6 +117,35 @@ int avggt_workspace_bytes(const avggt_params* p, size_t* build_ws_bytes, size_t*
 int avggt_build_kv(const avggt_params* p, const void* K, const void* V,
                    void* Kc, void* Vc, int32_t* idx, float* kmean, float* vmean,
                    void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * avggt_build_kv for callers that cannot allocate.  (The paper has no counterpart to this
+ * entry point; it exists for the sake of the library's users.)
+ *
+ * Who needs it: a program whose memory manager owns every byte of device memory before this
+ * library is loaded, a plugin that lives under another process's fixed memory budget, or a
+ * latency-critical loop that must not call cudaMalloc because it synchronises the device.
+ * Such a caller has no workspace to lend.  Here the scratch of the mean reduction (the
+ * per-block partial sums) is a fixed array inside the library image: about 2.3 MiB that every
+ * GPU which loads the library holds until the process exits.
+ *
+ * Same inputs, outputs and results as avggt_build_kv (the mean pair may differ in the last
+ * bits, because the partial sums are grouped over fewer blocks), with these differences:
+ *   - no ws / ws_bytes arguments; the call makes no cudaMalloc, cudaFree or other allocating
+ *     call, on any path;
+ *   - limit: n_heads * head_dim <= 1024.  Larger problems are rejected with
+ *     AVGGT_ERR_STATIC_SCRATCH before anything is enqueued;
+ *   - the first call on each device looks up the array's device address (and the device's
+ *     properties) with that device current; make that first call before any stream capture
+ *     begins.  Later calls only enqueue kernels;
+ *   - all calls on one device share the one array.  Each call rewrites every element it later
+ *     reads, so the previous call's contents do no harm and nothing needs clearing; but two
+ *     calls whose kernels overlap on the GPU (different streams, or different host threads)
+ *     race on it and give wrong means.  Serialise them on one stream.
+ */
+int avggt_build_kv_noalloc(const avggt_params* p, const void* K, const void* V,
+                           void* Kc, void* Vc, int32_t* idx, float* kmean, float* vmean,
+                           void* cuda_stream);
 
 /*
  * Subsampled global attention (Sec. 4.3): for every query token i and head h

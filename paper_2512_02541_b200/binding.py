@@ -17,13 +17,14 @@ AVGGT_ERR_WORKSPACE_TOO_SMALL = -3
 AVGGT_ERR_ALIGNMENT = -4
 AVGGT_ERR_CUDA = -5
 AVGGT_ERR_DEVICE_TIMEOUT = -6
+AVGGT_ERR_STATIC_SCRATCH = -7
 
 AVGGT_FLAG_KEEP_FIRST_FRAME = 1
 AVGGT_MEAN_OFF, AVGGT_MEAN_UNIT, AVGGT_MEAN_FILL = 0, 1, 2
 
 # every symbol include/avggt.h declares
 EXPORTS = (
-    "avggt_kv_count", "avggt_workspace_bytes", "avggt_build_kv", "avggt_global_attn",
+    "avggt_kv_count", "avggt_workspace_bytes", "avggt_build_kv", "avggt_build_kv_noalloc", "avggt_global_attn",
     "avggt_check_status", "avggt_strerror", "avggt_last_cuda_error", "avggt_version",
 )
 
@@ -78,6 +79,8 @@ def lib():
         L.avggt_kv_count.argtypes = [pp, i64p, i64p]
         L.avggt_workspace_bytes.argtypes = [pp, szp, szp]
         L.avggt_build_kv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.avggt_build_kv_noalloc.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.avggt_build_kv_noalloc.restype = ctypes.c_int
         L.avggt_global_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.avggt_check_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
         L.avggt_strerror.argtypes = [ctypes.c_int]
@@ -128,6 +131,16 @@ def avggt_build_kv(params, K, V, Kc, Vc, idx, kmean, vmean, ws, ws_bytes, stream
     """Enqueue the K/V compaction + mean reduction.  Arguments are tensors (or raw addresses)."""
     _check(lib().avggt_build_kv(ctypes.byref(params), _ptr(K), _ptr(V), _ptr(Kc), _ptr(Vc), _ptr(idx), _ptr(kmean),
                                 _ptr(vmean), _ptr(ws), ws_bytes, stream), "avggt_build_kv")
+
+
+def avggt_build_kv_noalloc(params, K, V, Kc, Vc, idx, kmean, vmean, stream=None):
+    """avggt_build_kv without a workspace, for callers that cannot allocate device memory (a host
+    whose memory manager owns the whole GPU, a plugin under a fixed budget, a loop that must not
+    call cudaMalloc).  The scratch is a fixed array inside the library: n_heads * head_dim <= 1024,
+    calls that overlap on the GPU race, and the first call on a device should precede any stream
+    capture.  This binding allocates nothing either."""
+    _check(lib().avggt_build_kv_noalloc(ctypes.byref(params), _ptr(K), _ptr(V), _ptr(Kc), _ptr(Vc), _ptr(idx),
+                                        _ptr(kmean), _ptr(vmean), stream), "avggt_build_kv_noalloc")
 
 
 def avggt_global_attn(params, Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws, ws_bytes, stream=None):

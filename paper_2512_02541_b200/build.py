@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libavggt.so")
-SOURCES = ["api.cu", "build_kv.cu", "global_attn.cu"]
+SOURCES = ["api.cu", "build_kv.cu", "build_kv_noalloc.cu", "global_attn.cu"]
 HEADERS = ["internal.h", "plan.h", "ptx.cuh", "tmap.h", os.path.join("..", "..", "include", "avggt.h")]
 
 

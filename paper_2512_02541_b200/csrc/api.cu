@@ -187,6 +187,7 @@ const char* avggt_strerror(int code) {
     case AVGGT_ERR_ALIGNMENT: return "device pointer not 16-byte aligned";
     case AVGGT_ERR_CUDA: return "CUDA call failed";
     case AVGGT_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+    case AVGGT_ERR_STATIC_SCRATCH: return "problem exceeds the fixed scratch of avggt_build_kv_noalloc (n_heads * head_dim <= 1024)";
     default: return "unknown error code";
   }
 }
