@@ -8,9 +8,10 @@
 //               through a ring of shared-memory stages (128-byte swizzle); the
 //               last two ring items are the K/V rows of the CTA's own queries
 //               (the preserved diagonal)
-//   warp  9     MMA issuer: S_t = Q_t Kc_j^T and O_t += P_t Vc_j with tcgen05.mma,
-//               bf16 operands, fp32 accumulators in tensor memory
-//   warps 10-11 idle (they complete the third warpgroup so that registers can
+//   warps 9-10  MMA issuers, one per query tile: S_t = Q_t Kc_j^T and
+//               O_t += P_t Vc_j with tcgen05.mma, bf16 operands, fp32
+//               accumulators in tensor memory
+//   warp  11    idle (it completes the third warpgroup so that registers can
 //               be moved to the softmax warpgroups)
 // Tensor memory per tile: S 128 columns (fp32), P 64 columns (bf16 pairs),
 // O 64 columns (fp32); 512 columns in all.  A softmax thread pulls its row of
@@ -47,6 +48,25 @@ constexpr uint32_t kColP = 128, kColO = 192;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 
+// Of every 8 pairs of scores, this many take their exponential from a polynomial on the FMA
+// pipe instead of the special-function unit (which, at 16 results per clock per SM, is the
+// scarcest resource of the softmax at head dimension 64).
+#ifndef AVGGT_POLY_EIGHTHS
+#define AVGGT_POLY_EIGHTHS 3
+#endif
+// 1: the two softmax warps that share a scheduler (one of each query tile) take turns in the
+// exponential phase, so that one warp's loads, maxima and stores run under the other's exponentials.
+#ifndef AVGGT_PINGPONG
+#define AVGGT_PINGPONG 1
+#endif
+// Columns per trip of the (rolled) exponential loop: 32, 64 or 128 (= fully unrolled).
+#ifndef AVGGT_CHUNK
+#define AVGGT_CHUNK 64
+#endif
+constexpr int kPolyEighths = AVGGT_POLY_EIGHTHS;
+constexpr int kChunk = AVGGT_CHUNK;
+static_assert(kChunk == 32 || kChunk == 64 || kChunk == 128, "chunk of the exponential loop");
+
 struct AttnArgs {
   Plan pl;
   const float* kmean;   // [H, d] or null
@@ -68,6 +88,7 @@ struct __align__(8) Barriers {
   uint64_t s_free[kQTiles];    // softmax -> MMA: S_t(j) has been read into registers
   uint64_t p_full[kQTiles];    // softmax -> MMA: P_t(j) stored (and O_t rescaled)
   uint64_t o_done[kQTiles];    // MMA -> softmax: P_t(j) V_j has completed
+  uint64_t turn[kQTiles][4];   // softmax warp w of the other tile -> warp w of this tile: the exponential unit is yours
   uint32_t tmem_base;
   uint32_t abort_flag;
 };
@@ -122,12 +143,20 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   return d;
 }
 
+// Register budget per thread after the roles have split.  The sum over all warps must not
+// exceed what the launch allocated (168 x 384): a setmaxnreg.inc that asks for more than the
+// pool can ever hold waits for ever, and that wait has no time limit.
+constexpr int kRegsSoftmax = 232, kRegsOther = 40;
+static_assert(kRegsSoftmax * kSoftmaxWarps + kRegsOther * (kThreads / 32 - kSoftmaxWarps) <= 168 * (kThreads / 32),
+              "register budget after setmaxnreg exceeds the launch allocation");
 template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
 // Optional per-phase cycle counters of the softmax loop (a tuning aid; compiled out by default).
 #ifdef AVGGT_PHASE_TIMERS
-__device__ unsigned long long g_phase_cycles[2][8];
+__device__ unsigned long long g_phase_cycles[2][4][8];   // [tile][warp of the tile][phase], CTA (0, 0)
+__device__ long long g_trace[64];
+#define AVGGT_TRACE(cond, slot) do { if ((cond) && blockIdx.x == 3 && blockIdx.y == 0) g_trace[slot] = clock64(); } while (0)
 struct PhaseTimers {
   unsigned long long acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
   long long last = 0;
@@ -135,6 +164,7 @@ struct PhaseTimers {
   __device__ __forceinline__ void lap(int i) { const long long now = clock64(); acc[i] += now - last; last = now; }
 };
 #else
+#define AVGGT_TRACE(cond, slot) do { } while (0)
 struct PhaseTimers {
   __device__ __forceinline__ void start() {}
   __device__ __forceinline__ void lap(int) {}
@@ -147,150 +177,252 @@ struct SmemLayout {
   uint8_t* v;   // kStages tiles
 };
 
-// ------------------------------------------------------------------ TMA producer (one thread)
+// The producer and the MMA issuers run with all 32 lanes of their warp in step (every branch
+// condition is made warp-uniform with a vote) and issue the TMA / tcgen05 instructions from one
+// elected lane.  Those instructions take their operands from the uniform datapath; issued from
+// divergent single-lane code they fall on a slow path that costs on the order of 100 clocks each.
+constexpr uint32_t kFullMask = 0xffffffffu;
+
+__device__ __forceinline__ bool wait_bar_warp(uint64_t* bar, uint32_t parity, Barriers* bars, const AttnArgs& a,
+                                              uint32_t where, uint32_t iter, bool check_abort = true) {
+  return __all_sync(kFullMask, wait_bar(bar, parity, bars, a, where, iter, check_abort));
+}
+
+// ------------------------------------------------------------------ TMA producer (one warp)
 __device__ __forceinline__ void producer_role(const CUtensorMap* tm_q, const CUtensorMap* tm_k, const CUtensorMap* tm_v,
                                               const CUtensorMap* tm_kc, const CUtensorMap* tm_vc, const AttnArgs& a,
                                               Barriers* bars, const SmemLayout& sm, int head, int q0) {
   const int n_kv = a.n_kv_tiles;
   const int n_items = n_kv + (a.use_diag ? kQTiles : 0);
-  mbar_arrive_expect_tx(smem_u32(&bars->q_full), kQTiles * kTileBytes);
+  if (elect_one()) {
+    prefetch_tensormap(tm_q);
+    prefetch_tensormap(tm_kc);
+    prefetch_tensormap(tm_vc);
+    mbar_arrive_expect_tx(smem_u32(&bars->q_full), kQTiles * kTileBytes);
 #pragma unroll
-  for (int t = 0; t < kQTiles; ++t)
-    tma_load_2d(smem_u32(sm.q[t]), tm_q, head * kHeadDim, q0 + t * kTileQ, smem_u32(&bars->q_full));
+    for (int t = 0; t < kQTiles; ++t)
+      tma_load_2d(smem_u32(sm.q[t]), tm_q, head * kHeadDim, q0 + t * kTileQ, smem_u32(&bars->q_full));
+  }
+  __syncwarp();
   int it = 0;
+  int stage = 0;
+  uint32_t empty_parity = 1;   // a fresh barrier passes the wait on the "previous" phase at once
   bool ok = true;
   for (; it < n_items; ++it) {
-    const int s = it % kStages;
-    const uint32_t round = static_cast<uint32_t>(it / kStages);
-    // a fresh barrier passes the wait on the "previous" phase at once
-    ok = wait_bar(&bars->k_empty[s], (round & 1) ^ 1, bars, a, 10, it);
+    ok = wait_bar_warp(&bars->k_empty[stage], empty_parity, bars, a, 10, it);
     if (!ok) break;
-    const uint32_t kb = smem_u32(&bars->k_full[s]);
-    mbar_arrive_expect_tx(kb, kTileBytes);
-    if (it < n_kv) tma_load_3d(smem_u32(sm.k + s * kTileBytes), tm_kc, 0, it * kTileKV, head, kb);
-    else tma_load_2d(smem_u32(sm.k + s * kTileBytes), tm_k, head * kHeadDim, q0 + (it - n_kv) * kTileQ, kb);
-    ok = wait_bar(&bars->v_empty[s], (round & 1) ^ 1, bars, a, 11, it);
+    if (elect_one()) {
+      const uint32_t kb = smem_u32(&bars->k_full[stage]);
+      mbar_arrive_expect_tx(kb, kTileBytes);
+      if (it < n_kv) tma_load_3d(smem_u32(sm.k + stage * kTileBytes), tm_kc, 0, it * kTileKV, head, kb);
+      else tma_load_2d(smem_u32(sm.k + stage * kTileBytes), tm_k, head * kHeadDim, q0 + (it - n_kv) * kTileQ, kb);
+    }
+    __syncwarp();
+    ok = wait_bar_warp(&bars->v_empty[stage], empty_parity, bars, a, 11, it);
     if (!ok) break;
-    const uint32_t vb = smem_u32(&bars->v_full[s]);
-    mbar_arrive_expect_tx(vb, kTileBytes);
-    if (it < n_kv) tma_load_3d(smem_u32(sm.v + s * kTileBytes), tm_vc, 0, it * kTileKV, head, vb);
-    else tma_load_2d(smem_u32(sm.v + s * kTileBytes), tm_v, head * kHeadDim, q0 + (it - n_kv) * kTileQ, vb);
+    if (elect_one()) {
+      const uint32_t vb = smem_u32(&bars->v_full[stage]);
+      mbar_arrive_expect_tx(vb, kTileBytes);
+      if (it < n_kv) tma_load_3d(smem_u32(sm.v + stage * kTileBytes), tm_vc, 0, it * kTileKV, head, vb);
+      else tma_load_2d(smem_u32(sm.v + stage * kTileBytes), tm_v, head * kHeadDim, q0 + (it - n_kv) * kTileQ, vb);
+    }
+    __syncwarp();
+    if (++stage == kStages) { stage = 0; empty_parity ^= 1; }
   }
   if (!ok) {
     // let the copies still in flight land before the CTA gives up its shared memory
-    (void)wait_bar(&bars->q_full, 0, bars, a, 12, 0, false);
+    (void)wait_bar_warp(&bars->q_full, 0, bars, a, 12, 0, false);
     for (int back = 1; back <= kStages && it - back >= 0; ++back) {
       const int jt = it - back;
-      (void)wait_bar(&bars->k_full[jt % kStages], (jt / kStages) & 1, bars, a, 12, jt, false);
-      (void)wait_bar(&bars->v_full[jt % kStages], (jt / kStages) & 1, bars, a, 12, jt, false);
+      (void)wait_bar_warp(&bars->k_full[jt % kStages], (jt / kStages) & 1, bars, a, 12, jt, false);
+      (void)wait_bar_warp(&bars->v_full[jt % kStages], (jt / kStages) & 1, bars, a, 12, jt, false);
     }
   }
 }
 
-// ------------------------------------------------------------------ MMA issuer (one thread)
-__device__ __forceinline__ void mma_role(const AttnArgs& a, Barriers* bars, const SmemLayout& sm, uint32_t tmem) {
-  const int n_kv = a.n_kv_tiles;
-  const uint32_t idesc_qk = umma_idesc_bf16(kTileQ, kTileKV, false);
-  const uint32_t idesc_pv = umma_idesc_bf16(kTileQ, kHeadDim, true);
-  uint64_t desc_q[kQTiles];
-#pragma unroll
-  for (int t = 0; t < kQTiles; ++t) desc_q[t] = umma_desc_sw128(smem_u32(sm.q[t]));
-
-  auto issue_qk = [&](int t, int j) {
-    const uint64_t desc_k = umma_desc_sw128(smem_u32(sm.k + (j % kStages) * kTileBytes));
+// ------------------------------------------------------------------ MMA issuer (one warp per query tile)
+// Per tile the order of events is fixed: S_t(j) is read by the softmax (s_free) before P_t(j) is
+// stored (p_full), which precedes the read of S_t(j+1).  The issuer of tile t therefore waits, in
+// turn, for "S_t free and K_{j+1} loaded" -> Q K^T of step j+1, then "P_t(j) stored and V_j
+// loaded" -> P V of step j.  A K or V stage is released when both tiles' issuers have committed
+// their product on it (the empty barriers count two arrivals).
+template <int t>
+__device__ __forceinline__ void issue_qk(const AttnArgs& a, Barriers* bars, uint32_t tmem, uint64_t desc_q, uint32_t k_base,
+                                         int stage, int j) {
+  if (elect_one()) {
+    constexpr uint32_t idesc = umma_idesc_bf16(kTileQ, kTileKV, false);
+    const uint64_t desc_k = umma_desc_sw128(k_base + stage * kTileBytes);
+    AVGGT_TRACE(j == 101, 16 + t);
 #pragma unroll
     for (int k = 0; k < kHeadDim / 16; ++k)
-      umma_ss(tmem + t * kTmemTileStride, desc_q[t] + (k * 32 >> 4), desc_k + (k * 32 >> 4), idesc_qk, k > 0);
+      umma_ss(tmem + t * kTmemTileStride, desc_q + (k * 32 >> 4), desc_k + (k * 32 >> 4), idesc, k > 0);
     umma_commit(smem_u32(&bars->s_full[t]));
-  };
-  auto issue_pv = [&](int t, int j) {
-    const uint64_t desc_v = umma_desc_sw128(smem_u32(sm.v + (j % kStages) * kTileBytes));
+    umma_commit(smem_u32(&bars->k_empty[stage]));
+  }
+  __syncwarp();
+}
+
+template <int t>
+__device__ __forceinline__ void issue_pv(const AttnArgs& a, Barriers* bars, uint32_t tmem, uint32_t v_base, int stage, int j) {
+  if (elect_one()) {
+    constexpr uint32_t idesc = umma_idesc_bf16(kTileQ, kHeadDim, true);
+    const uint64_t desc_v = umma_desc_sw128(v_base + stage * kTileBytes);
+    AVGGT_TRACE(j == 100, 18 + t);
 #pragma unroll
     for (int k = 0; k < kTileKV / 16; ++k)
       umma_ts(tmem + t * kTmemTileStride + kColO, tmem + t * kTmemTileStride + kColP + k * 8, desc_v + (k * 2048 >> 4),
-              idesc_pv, (j > 0 || k > 0) ? 1u : 0u);
+              idesc, (j > 0 || k > 0) ? 1u : 0u);
     umma_commit(smem_u32(&bars->o_done[t]));
-  };
+    umma_commit(smem_u32(&bars->v_empty[stage]));
+  }
+  __syncwarp();
+}
 
-  if (!wait_bar(&bars->q_full, 0, bars, a, 20, 0)) return;
-  if (!wait_bar(&bars->k_full[0], 0, bars, a, 21, 0)) return;
+template <int t>
+__device__ __forceinline__ void mma_role(const AttnArgs& a, Barriers* bars, const SmemLayout& sm, uint32_t tmem) {
+  static_assert(kStages >= 2, "the K ring must hold the tile in use and the next one");
+  const int n_kv = a.n_kv_tiles;
+  const uint64_t desc_q = umma_desc_sw128(smem_u32(sm.q[t]));
+  const uint32_t k_base = smem_u32(sm.k), v_base = smem_u32(sm.v);
+
+  if (!wait_bar_warp(&bars->q_full, 0, bars, a, 20, 0)) return;
+  if (!wait_bar_warp(&bars->k_full[0], 0, bars, a, 21, 0)) return;
   tc_fence_after();
-#pragma unroll
-  for (int t = 0; t < kQTiles; ++t) issue_qk(t, 0);
-  umma_commit(smem_u32(&bars->k_empty[0]));
+  issue_qk<t>(a, bars, tmem, desc_q, k_base, 0, 0);
 
-  // Event loop: issue whichever product has its operands ready.  Per tile, Q K^T of step j
-  // needs S_t free (softmax read step j-1) and K_j; P V of step j needs P_t(j) and V_j.
-  // No barrier polled here can be more than one phase ahead of the step it is polled for.
-  static_assert(kQTiles == 2, "the issue loop below is written for two query tiles");
-  int qk0 = 1, qk1 = 1, pv0 = 0, pv1 = 0;   // next step to issue, per tile
-  uint64_t t_idle = 0;
-  uint32_t idle_polls = 0;
-  bool progressed;
-  auto poll_tile = [&](int t, int& qk_mine, int& pv_mine, const int& qk_other, const int& pv_other) {
-    const int jq = qk_mine;
-    if (jq < n_kv && mbar_test_wait(smem_u32(&bars->s_free[t]), (jq - 1) & 1) &&
-        mbar_test_wait(smem_u32(&bars->k_full[jq % kStages]), (jq / kStages) & 1)) {
+  int k_stage = 1, v_stage = 0;          // stage of K_{j+1} and of V_j
+  uint32_t k_parity = 0, v_parity = 0;   // parity of their "full" phase
+  for (int j = 0; j < n_kv; ++j) {
+    if (j + 1 < n_kv) {
+      AVGGT_TRACE(j == 100 && elect_one(), 40 + t);
+      if (!wait_bar_warp(&bars->s_free[t], j & 1, bars, a, 22 + t, j)) return;
+      AVGGT_TRACE(j == 100 && elect_one(), 42 + t);
+      if (!wait_bar_warp(&bars->k_full[k_stage], k_parity, bars, a, 24 + t, j)) return;
       tc_fence_after();
-      issue_qk(t, jq);
-      qk_mine = jq + 1;
-      if (qk_other > jq) umma_commit(smem_u32(&bars->k_empty[jq % kStages]));   // both tiles have read K_jq
-      progressed = true;
+      issue_qk<t>(a, bars, tmem, desc_q, k_base, k_stage, j + 1);
+      if (++k_stage == kStages) { k_stage = 0; k_parity ^= 1; }
     }
-    const int jp = pv_mine;
-    if (jp < n_kv && mbar_test_wait(smem_u32(&bars->p_full[t]), jp & 1) &&
-        mbar_test_wait(smem_u32(&bars->v_full[jp % kStages]), (jp / kStages) & 1)) {
-      tc_fence_after();
-      issue_pv(t, jp);
-      pv_mine = jp + 1;
-      if (pv_other > jp) umma_commit(smem_u32(&bars->v_empty[jp % kStages]));   // both tiles have read V_jp
-      progressed = true;
-    }
-  };
-  while (true) {
-    progressed = false;
-    poll_tile(0, qk0, pv0, qk1, pv1);
-    poll_tile(1, qk1, pv1, qk0, pv0);
-    const bool finished = pv0 >= n_kv && pv1 >= n_kv;
-    if (finished) break;
-    if (progressed) { idle_polls = 0; continue; }
-    if ((++idle_polls & 0xffu) == 0) {
-      if (*reinterpret_cast<volatile uint32_t*>(&bars->abort_flag)) return;
-      const uint64_t now = globaltimer_ns();
-      if (idle_polls == 0x100u) t_idle = now;
-      else if (now - t_idle > AVGGT_WAIT_LIMIT_NS) { report_timeout(a, bars, 26, pv0); return; }
-    }
+    AVGGT_TRACE(j == 100 && elect_one(), 46 + t);
+    if (!wait_bar_warp(&bars->p_full[t], j & 1, bars, a, 26 + t, j)) return;
+    AVGGT_TRACE(j == 100 && elect_one(), 48 + t);
+    if (!wait_bar_warp(&bars->v_full[v_stage], v_parity, bars, a, 28 + t, j)) return;
+    tc_fence_after();
+    issue_pv<t>(a, bars, tmem, v_base, v_stage, j);
+    if (++v_stage == kStages) { v_stage = 0; v_parity ^= 1; }
   }
 }
 
 // ------------------------------------------------------------------ softmax warpgroup (128 threads per tile)
-// kLse: also keep the sum of the unrounded exponentials, for the log-sum-exp output.
-template <bool kMasked, bool kLse>
+// 2^x for a pair of values on the FMA pipe.  x = n + r with n = round(x), |r| <= 1/2: adding
+// 1.5 * 2^23 leaves n in the low mantissa bits of the sum; 2^r is a degree-3 minimax polynomial
+// (relative error 7.5e-5, a twenty-sixth of the bf16 rounding step the result goes through);
+// 2^n is applied by adding n to the exponent field.  Valid for x <= 100; x is clamped at -125.
+__device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1) {
+  float x0, x1;
+  unpack_f32x2(x2, x0, x1);
+  x2 = pack_f32x2(fmaxf(x0, -125.0f), fmaxf(x1, -125.0f));
+  const uint64_t magic = pack_f32x2(12582912.0f, 12582912.0f);
+  const uint64_t t = add_f32x2(x2, magic);
+  const uint64_t r = sub_f32x2(x2, sub_f32x2(t, magic));
+  uint64_t q = fma_f32x2(pack_f32x2(0x1.c3f76p-5f, 0x1.c3f76p-5f), r, pack_f32x2(0x1.f0de1ap-3f, 0x1.f0de1ap-3f));
+  q = fma_f32x2(q, r, pack_f32x2(0x1.62f31ap-1f, 0x1.62f31ap-1f));
+  q = fma_f32x2(q, r, pack_f32x2(0x1.fff692p-1f, 0x1.fff692p-1f));
+  float t0, t1, q0, q1;
+  unpack_f32x2(t, t0, t1);
+  unpack_f32x2(q, q0, q1);
+  p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
+  p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
+}
+
+// pair g (0..7 within a group of eight) goes to the polynomial when kPoly of eight do
+template <int kPoly>
+__device__ __forceinline__ constexpr bool pair_uses_poly(int g) { return ((g + 1) * kPoly) / 8 != (g * kPoly) / 8; }
+
+// First half of the work on sixteen scores of one query row (eight pairs, s[s0 .. s0+16)): scale,
+// subtract the reference maximum (folded into neg_m2) and start the exponentials; e[] receives
+// the results.
+template <int kPoly>
+__device__ __forceinline__ void softmax_issue16(const uint32_t (&s)[128], int s0, uint64_t scale2, uint64_t neg_m2,
+                                                float (&e)[16]) {
+  // the special-function unit first, so that it works through its queue while the polynomials run
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    if (!pair_uses_poly<kPoly>(i)) {
+      const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[s0 + 2 * i]), __uint_as_float(s[s0 + 2 * i + 1])), scale2, neg_m2);
+      float x0, x1;
+      unpack_f32x2(x2, x0, x1);
+      e[2 * i] = ex2_approx_inorder(x0);
+      e[2 * i + 1] = ex2_approx_inorder(x1);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    if (pair_uses_poly<kPoly>(i)) {
+      const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[s0 + 2 * i]), __uint_as_float(s[s0 + 2 * i + 1])), scale2, neg_m2);
+      exp2_poly_pair(x2, e[2 * i], e[2 * i + 1]);
+    }
+  }
+}
+
+// Second half, one block later (the exponentials have long landed): round to bf16 into
+// pk[0..8) and add to the sums for the normaliser (of the rounded values) and for the
+// log-sum-exp (unrounded).
+template <bool kLse>
+__device__ __forceinline__ void softmax_finish16(const float (&e)[16], uint64_t& sum2, uint64_t& sum_exact2, uint32_t (&pk)[8]) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const uint32_t w = pack_bf16x2(e[2 * i], e[2 * i + 1]);
+    pk[i] = w;
+    if (kLse) sum_exact2 = add_f32x2(sum_exact2, pack_f32x2(e[2 * i], e[2 * i + 1]));
+    sum2 = add_f32x2(sum2, pack_f32x2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)));
+  }
+}
+
+// One step of the online softmax of a query row: S_t(j) in tensor memory -> P_t(j) in tensor
+// memory, running reference maximum and sums updated.
+//
+// The row's 128 scores are pulled into registers at once and S_t is released, so that the next
+// Q K^T runs under this step's exponentials.  After the row maximum, the exponentials are taken
+// in a loop over chunks of kChunk columns that is kept rolled on purpose: fully unrolled, the
+// 128 exponentials of a row are thousands of instructions of straight-line code per step, and
+// the warps then run at the speed of instruction fetch, not of the exponential unit.
+// Registers cannot be indexed by a loop counter, so each trip works on the first kChunk
+// registers and then moves the rest down.  Within the loop the work is software-pipelined by
+// hand over blocks of 16 columns: a block's exponentials are rounded and summed only after the
+// next block's have been issued, so that no instruction waits on the unit's latency.
+// kPoly: pairs per eight whose exponential is a polynomial.  kLse: also keep the sum of the
+// unrounded exponentials, for the log-sum-exp output.  kMasked: columns >= valid are excluded.
+template <bool kMasked, bool kLse, int kPoly>
 __device__ __forceinline__ void softmax_step(uint32_t tS, uint32_t tP, uint32_t tO, int j, int valid, float scale_log2,
                                              float& m_used, float& l_run, float& l_exact, Barriers* bars,
-                                             const AttnArgs& a, int t, int lane, bool& ok, PhaseTimers& pt) {
-  uint32_t s[4][32];
-  tmem_ld32(tS, s[0]);
-  tmem_ld32(tS + 32, s[1]);
-  tmem_ld32(tS + 64, s[2]);
-  tmem_ld32(tS + 96, s[3]);
+                                             const AttnArgs& a, int t, int warp_in_tile, int lane, bool& ok,
+                                             PhaseTimers& pt) {
+  uint32_t s[128];
+  {
+    uint32_t (&s4)[4][32] = reinterpret_cast<uint32_t (&)[4][32]>(s);
+    tmem_ld32(tS, s4[0]);
+    tmem_ld32(tS + 32, s4[1]);
+    tmem_ld32(tS + 64, s4[2]);
+    tmem_ld32(tS + 96, s4[3]);
+  }
   tmem_wait_ld();
   tc_fence_before();
   __syncwarp();
   if (lane == 0) mbar_arrive(smem_u32(&bars->s_free[t]));
   pt.lap(1);
+  AVGGT_TRACE(j == 100 && warp_in_tile == 0 && lane == 0, t * 8 + 1);
 
   if (kMasked) {
 #pragma unroll
     for (int i = 0; i < 128; ++i)
-      if (i >= valid) s[i >> 5][i & 31] = __float_as_uint(-INFINITY);
+      if (i >= valid) s[i] = __float_as_uint(-INFINITY);
   }
   float mx[4];
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
-    mx[c] = fmaxf(__uint_as_float(s[c][0]), __uint_as_float(s[c][1]));
+    mx[c] = fmaxf(__uint_as_float(s[32 * c]), __uint_as_float(s[32 * c + 1]));
 #pragma unroll
-    for (int i = 2; i < 32; i += 2) mx[c] = max3(mx[c], __uint_as_float(s[c][i]), __uint_as_float(s[c][i + 1]));
+    for (int i = 2; i < 32; i += 2) mx[c] = max3(mx[c], __uint_as_float(s[32 * c + i]), __uint_as_float(s[32 * c + i + 1]));
   }
   const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;
   // lazy rescale: keep the old reference maximum unless the new one is far above it
@@ -304,53 +436,78 @@ __device__ __forceinline__ void softmax_step(uint32_t tS, uint32_t tP, uint32_t 
   }
   const bool rescale = (j > 0) && __any_sync(0xffffffffu, jump);
   pt.lap(2);
+  AVGGT_TRACE(j == 100 && warp_in_tile == 0 && lane == 0, t * 8 + 2);
 
-  // exponentials, rounded to bf16 for the value product; the normaliser sums the
-  // rounded values so that numerator and denominator carry the same weights
-  const float neg_m = -m_used;
-  float sum0 = 0.f, sum1 = 0.f, sum_exact = 0.f;
-  uint32_t pk[4][16];
-#pragma unroll
-  for (int c = 0; c < 4; ++c) {
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const float p0 = ex2_approx(fmaf(__uint_as_float(s[c][2 * i]), scale_log2, neg_m));
-      const float p1 = ex2_approx(fmaf(__uint_as_float(s[c][2 * i + 1]), scale_log2, neg_m));
-      const uint32_t w = pack_bf16x2(p0, p1);
-      pk[c][i] = w;
-      if (kLse) sum_exact += p0 + p1;
-      sum0 += __uint_as_float(w << 16);
-      sum1 += __uint_as_float(w & 0xffff0000u);
-    }
-  }
-
-  pt.lap(3);
   // P_t(j-1) must have been consumed, and O_t be at rest, before either is written
   if (j > 0) {
     if (!wait_bar(&bars->o_done[t], (j - 1) & 1, bars, a, 30 + t, j)) { ok = false; return; }
     tc_fence_after();
   }
-  pt.lap(4);
   if (rescale) {
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
+#pragma unroll 1
+    for (int h = 0; h < 2; ++h) {
       uint32_t o[32];
-      tmem_ld32(tO + c * 32, o);
+      tmem_ld32(tO + h * 32, o);
       tmem_wait_ld();
 #pragma unroll
       for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-      tmem_st32(tO + c * 32, o);
+      tmem_st32(tO + h * 32, o);
     }
   }
+  pt.lap(3);
+#if AVGGT_PINGPONG
+  // my turn on the exponential unit: the partner warp (same scheduler, other tile) has left its phase
+  if (!wait_bar(&bars->turn[t][warp_in_tile], j & 1, bars, a, 60 + t, j)) { ok = false; return; }
+#endif
+  pt.lap(4);
+  AVGGT_TRACE(j == 100 && warp_in_tile == 0 && lane == 0, t * 8 + 3);
+
+  // exponentials, rounded to bf16 for the value product; the normaliser sums the
+  // rounded values so that numerator and denominator carry the same weights
+  const uint64_t scale2 = pack_f32x2(scale_log2, scale_log2);
+  const uint64_t neg_m2 = pack_f32x2(-m_used, -m_used);
+  uint64_t sum2 = pack_f32x2(0.f, 0.f), sum_exact2 = pack_f32x2(0.f, 0.f);
+  constexpr int kBlocks = kChunk / 16;   // blocks of 16 columns per trip
+  float e[2][16];                        // exponentials in flight: block b uses e[b & 1]
+  uint32_t pk[8];                        // P of one block (16 columns as bf16 pairs)
+#pragma unroll 1
+  for (int c = 0; c < 128 / kChunk; ++c) {
 #pragma unroll
-  for (int c = 0; c < 4; ++c) tmem_st16(tP + c * 16, pk[c]);
-  l_run += sum0 + sum1;
-  if (kLse) l_exact += sum_exact;
+    for (int b = 0; b < kBlocks; ++b) {
+      softmax_issue16<kPoly>(s, 16 * b, scale2, neg_m2, e[b & 1]);
+      // round, sum and store the block before this one (the last block of the previous trip when b = 0)
+      if (b > 0 || c > 0) {
+        softmax_finish16<kLse>(e[(b & 1) ^ 1], sum2, sum_exact2, pk);
+        tmem_st8(tP + c * (kChunk / 2) + b * 8 - 8, pk);
+      }
+    }
+    if (kChunk < 128) {
+#pragma unroll
+      for (int i = 0; i < 128 - kChunk; ++i) s[i] = s[i + kChunk];
+    }
+  }
+  softmax_finish16<kLse>(e[1], sum2, sum_exact2, pk);
+  tmem_st8(tP + 56, pk);
+#if AVGGT_PINGPONG
+  __syncwarp();
+  if (lane == 0) mbar_arrive(smem_u32(&bars->turn[t ^ 1][warp_in_tile]));
+#endif
+  pt.lap(5);
+  AVGGT_TRACE(j == 100 && warp_in_tile == 0 && lane == 0, t * 8 + 4);
+
+  float sum_a, sum_b;
+  unpack_f32x2(sum2, sum_a, sum_b);
+  l_run += sum_a + sum_b;
+  if (kLse) {
+    unpack_f32x2(sum_exact2, sum_a, sum_b);
+    l_exact += sum_a + sum_b;
+  }
   tmem_wait_st();
   tc_fence_before();
   __syncwarp();
   if (lane == 0) mbar_arrive(smem_u32(&bars->p_full[t]));
-  pt.lap(5);
+  pt.lap(6);
+  AVGGT_TRACE(j == 100 && warp_in_tile == 0 && lane == 0, t * 8 + 6);
 }
 
 __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, const SmemLayout& sm, uint32_t tmem,
@@ -368,20 +525,28 @@ __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, 
   bool ok = true;
   PhaseTimers pt;
   pt.start();
+#if AVGGT_PINGPONG
+  // tile 0 goes first: tile 1 hands it the first turn
+  if (t == 1 && lane == 0) mbar_arrive(smem_u32(&bars->turn[0][wg_tid >> 5]));
+#endif
 
+#pragma unroll 1
   for (int j = 0; j < n_kv && ok; ++j) {
     if (!wait_bar(&bars->s_full[t], j & 1, bars, a, 40 + t, j)) { ok = false; break; }
     tc_fence_after();
     pt.lap(0);
+    AVGGT_TRACE(j == 100 && wg_tid == 0, t * 8 + 0);
+    AVGGT_TRACE(j == 101 && wg_tid == 0, t * 8 + 7);
     const int valid = static_cast<int>(pl.M - static_cast<int64_t>(j) * kTileKV);
-    if (valid < kTileKV) softmax_step<true, true>(tS, tP, tO, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, a, t, lane, ok, pt);
-    else if (want_lse) softmax_step<false, true>(tS, tP, tO, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, a, t, lane, ok, pt);
-    else softmax_step<false, false>(tS, tP, tO, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, a, t, lane, ok, pt);
+    // the masked (last, ragged) tile keeps every exponential on the special-function unit, where -inf gives an exact 0
+    if (valid < kTileKV) softmax_step<true, true, 0>(tS, tP, tO, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, a, t, wg_tid >> 5, lane, ok, pt);
+    else if (want_lse) softmax_step<false, true, kPolyEighths>(tS, tP, tO, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, a, t, wg_tid >> 5, lane, ok, pt);
+    else softmax_step<false, false, kPolyEighths>(tS, tP, tO, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, a, t, wg_tid >> 5, lane, ok, pt);
   }
   if (!ok) return;
 #ifdef AVGGT_PHASE_TIMERS
-  if (blockIdx.x == 0 && blockIdx.y == 0 && wg_tid == 0)
-    for (int i = 0; i < 8; ++i) g_phase_cycles[t][i] = pt.acc[i];
+  if (blockIdx.x == 0 && blockIdx.y == 0 && lane == 0)
+    for (int i = 0; i < 8; ++i) g_phase_cycles[t][wg_tid >> 5][i] = pt.acc[i];
 #endif
 
   // ---- epilogue: diagonal and mean-fill terms, normalisation, store
@@ -495,23 +660,27 @@ global_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   __shared__ Barriers bars;
 
   const int tid = threadIdx.x;
-  const int warp = tid >> 5;
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // warp-uniform by construction
   const int head = blockIdx.y;
   const int q0 = blockIdx.x * (kQTiles * kTileQ);
+
+  // a launch in which a wait has already run out is abandoned: the remaining CTAs leave at once
+  if (__syncthreads_or(*reinterpret_cast<volatile uint32_t*>(a.status) != 0u)) return;
 
   if (tid == 0) {
     mbar_init(smem_u32(&bars.q_full), 1);
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&bars.k_full[s]), 1);
-      mbar_init(smem_u32(&bars.k_empty[s]), 1);
+      mbar_init(smem_u32(&bars.k_empty[s]), kQTiles);
       mbar_init(smem_u32(&bars.v_full[s]), 1);
-      mbar_init(smem_u32(&bars.v_empty[s]), 1);
+      mbar_init(smem_u32(&bars.v_empty[s]), kQTiles);
     }
     for (int t = 0; t < kQTiles; ++t) {
       mbar_init(smem_u32(&bars.s_full[t]), 1);
       mbar_init(smem_u32(&bars.s_free[t]), 4);
       mbar_init(smem_u32(&bars.p_full[t]), 4);
       mbar_init(smem_u32(&bars.o_done[t]), 1);
+      for (int w = 0; w < 4; ++w) mbar_init(smem_u32(&bars.turn[t][w]), 1);
     }
     bars.abort_flag = 0;
     fence_mbar_init();
@@ -526,21 +695,14 @@ global_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const uint32_t tmem = bars.tmem_base;
 
   if (warp < kSoftmaxWarps) {
-    reg_inc<224>();
+    reg_inc<kRegsSoftmax>();
     const int t = warp >> 2;
     softmax_role(a, &bars, sm, tmem, t, tid & 127, head, q0);
   } else {
-    reg_dec<56>();
-    if (warp == kTmaWarp) {
-      if ((tid & 31) == 0) {
-        prefetch_tensormap(&tm_q);
-        prefetch_tensormap(&tm_kc);
-        prefetch_tensormap(&tm_vc);
-        producer_role(&tm_q, &tm_k, &tm_v, &tm_kc, &tm_vc, a, &bars, sm, head, q0);
-      }
-    } else if (warp == kMmaWarp) {
-      if ((tid & 31) == 0) mma_role(a, &bars, sm, tmem);
-    }
+    reg_dec<kRegsOther>();
+    if (warp == kTmaWarp) producer_role(&tm_q, &tm_k, &tm_v, &tm_kc, &tm_vc, a, &bars, sm, head, q0);
+    else if (warp == kMmaWarp) mma_role<0>(a, &bars, sm, tmem);
+    else if (warp == kMmaWarp + 1) mma_role<1>(a, &bars, sm, tmem);
   }
 
   tc_fence_before();
@@ -553,6 +715,16 @@ constexpr size_t kAttnSmemBytes = static_cast<size_t>(kTileBytes) * (kQTiles + 2
 }  // namespace
 
 size_t global_attn_ws_bytes(const Plan&, int) { return kAttnStatusBytes; }
+
+#ifdef AVGGT_PHASE_TIMERS
+// Tuning aids: copy the 2 x 4 x 8 phase counters / the 64 event stamps of the last launch to the host.
+extern "C" int avggt_debug_phase_cycles(unsigned long long* out64) {
+  return cudaMemcpyFromSymbol(out64, g_phase_cycles, sizeof(g_phase_cycles)) == cudaSuccess ? 0 : -1;
+}
+extern "C" int avggt_debug_trace(long long* out64) {
+  return cudaMemcpyFromSymbol(out64, g_trace, sizeof(g_trace)) == cudaSuccess ? 0 : -1;
+}
+#endif
 
 cudaError_t launch_global_attn(const Plan& pl, int /*sm_count*/, const void* Q, const void* K, const void* V,
                                const void* Kc, const void* Vc, const float* kmean, const float* vmean, void* O,
