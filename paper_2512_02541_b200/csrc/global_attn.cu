@@ -52,20 +52,19 @@ constexpr float kRescaleThreshold = 8.0f;   // log2 units
 // pipe instead of the special-function unit (which, at 16 results per clock per SM, is the
 // scarcest resource of the softmax at head dimension 64).
 #ifndef AVGGT_POLY_EIGHTHS
-#define AVGGT_POLY_EIGHTHS 3
+#define AVGGT_POLY_EIGHTHS 2
 #endif
 // 1: the two softmax warps that share a scheduler (one of each query tile) take turns in the
 // exponential phase, so that one warp's loads, maxima and stores run under the other's exponentials.
 #ifndef AVGGT_PINGPONG
-#define AVGGT_PINGPONG 1
-#endif
-// Columns per trip of the (rolled) exponential loop: 32, 64 or 128 (= fully unrolled).
-#ifndef AVGGT_CHUNK
-#define AVGGT_CHUNK 64
+#define AVGGT_PINGPONG 0
 #endif
 constexpr int kPolyEighths = AVGGT_POLY_EIGHTHS;
-constexpr int kChunk = AVGGT_CHUNK;
-static_assert(kChunk == 32 || kChunk == 64 || kChunk == 128, "chunk of the exponential loop");
+// How many pairs the rounding and summing of the exponentials trails their issue.
+#ifndef AVGGT_EXP_LAG
+#define AVGGT_EXP_LAG 3
+#endif
+constexpr int kExpLag = AVGGT_EXP_LAG;
 
 struct AttnArgs {
   Plan pl;
@@ -338,43 +337,47 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1
 template <int kPoly>
 __device__ __forceinline__ constexpr bool pair_uses_poly(int g) { return ((g + 1) * kPoly) / 8 != (g * kPoly) / 8; }
 
-// First half of the work on sixteen scores of one query row (eight pairs, s[s0 .. s0+16)): scale,
-// subtract the reference maximum (folded into neg_m2) and start the exponentials; e[] receives
-// the results.
-template <int kPoly>
-__device__ __forceinline__ void softmax_issue16(const uint32_t (&s)[128], int s0, uint64_t scale2, uint64_t neg_m2,
-                                                float (&e)[16]) {
-  // the special-function unit first, so that it works through its queue while the polynomials run
+// The 128 scores of one query row -> bf16 probabilities, stored to tensor memory at tP as they
+// are produced, relative to the reference maximum folded into neg_m2; adds to the sums for the
+// normaliser (of the rounded values) and for the log-sum-exp (unrounded).
+//
+// A warp issues in order, and an exponential holds the special-function unit for 8 clocks, so
+// the exponentials are spaced out by hand: between two of them sit the scaling of the next pair
+// and the rounding and summing of the pair issued kExpLag pairs earlier (whose results have
+// landed by then).  The "_inorder" instructions are volatile, which keeps them in this order.
+template <bool kLse, int kPoly>
+__device__ __forceinline__ void softmax_row(const uint32_t (&s)[128], uint64_t scale2, uint64_t neg_m2, uint64_t& sum2,
+                                            uint64_t& sum_exact2, uint32_t tP) {
+  float e0[64], e1[64];   // indexed statically: only the pairs in flight occupy registers
+  uint32_t pk[8];         // P of 16 columns as bf16 pairs
+  uint64_t x2_next = fma_f32x2_inorder(pack_f32x2(__uint_as_float(s[0]), __uint_as_float(s[1])), scale2, neg_m2);
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    if (!pair_uses_poly<kPoly>(i)) {
-      const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[s0 + 2 * i]), __uint_as_float(s[s0 + 2 * i + 1])), scale2, neg_m2);
-      float x0, x1;
-      unpack_f32x2(x2, x0, x1);
-      e[2 * i] = ex2_approx_inorder(x0);
-      e[2 * i + 1] = ex2_approx_inorder(x1);
+  for (int i = 0; i < 64 + kExpLag; ++i) {
+    const int k = i - kExpLag;   // the pair that is rounded and summed in this slot
+    float x1 = 0.f;
+    bool mufu = false;
+    if (i < 64) {
+      const uint64_t x2 = x2_next;
+      if (i + 1 < 64)
+        x2_next = fma_f32x2_inorder(pack_f32x2(__uint_as_float(s[2 * i + 2]), __uint_as_float(s[2 * i + 3])), scale2, neg_m2);
+      if (pair_uses_poly<kPoly>(i & 7)) {
+        exp2_poly_pair(x2, e0[i], e1[i]);
+      } else {
+        float x0;
+        unpack_f32x2(x2, x0, x1);
+        e0[i] = ex2_approx_inorder(x0);
+        mufu = true;
+      }
     }
-  }
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    if (pair_uses_poly<kPoly>(i)) {
-      const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[s0 + 2 * i]), __uint_as_float(s[s0 + 2 * i + 1])), scale2, neg_m2);
-      exp2_poly_pair(x2, e[2 * i], e[2 * i + 1]);
+    uint32_t w = 0;
+    if (k >= 0) w = pack_bf16x2_inorder(e0[k], e1[k]);
+    if (mufu) e1[i] = ex2_approx_inorder(x1);
+    if (k >= 0) {
+      pk[k & 7] = w;
+      if (kLse) sum_exact2 = add_f32x2(sum_exact2, pack_f32x2(e0[k], e1[k]));
+      sum2 = add_f32x2(sum2, pack_f32x2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)));
+      if ((k & 7) == 7) tmem_st8(tP + (k >> 3) * 8, pk);
     }
-  }
-}
-
-// Second half, one block later (the exponentials have long landed): round to bf16 into
-// pk[0..8) and add to the sums for the normaliser (of the rounded values) and for the
-// log-sum-exp (unrounded).
-template <bool kLse>
-__device__ __forceinline__ void softmax_finish16(const float (&e)[16], uint64_t& sum2, uint64_t& sum_exact2, uint32_t (&pk)[8]) {
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const uint32_t w = pack_bf16x2(e[2 * i], e[2 * i + 1]);
-    pk[i] = w;
-    if (kLse) sum_exact2 = add_f32x2(sum_exact2, pack_f32x2(e[2 * i], e[2 * i + 1]));
-    sum2 = add_f32x2(sum2, pack_f32x2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)));
   }
 }
 
@@ -382,14 +385,8 @@ __device__ __forceinline__ void softmax_finish16(const float (&e)[16], uint64_t&
 // memory, running reference maximum and sums updated.
 //
 // The row's 128 scores are pulled into registers at once and S_t is released, so that the next
-// Q K^T runs under this step's exponentials.  After the row maximum, the exponentials are taken
-// in a loop over chunks of kChunk columns that is kept rolled on purpose: fully unrolled, the
-// 128 exponentials of a row are thousands of instructions of straight-line code per step, and
-// the warps then run at the speed of instruction fetch, not of the exponential unit.
-// Registers cannot be indexed by a loop counter, so each trip works on the first kChunk
-// registers and then moves the rest down.  Within the loop the work is software-pipelined by
-// hand over blocks of 16 columns: a block's exponentials are rounded and summed only after the
-// next block's have been issued, so that no instruction waits on the unit's latency.
+// Q K^T runs under this step's exponentials.  The row maximum decides whether the reference
+// maximum moves (lazy rescale); then softmax_row takes the exponentials.
 // kPoly: pairs per eight whose exponential is a polynomial.  kLse: also keep the sum of the
 // unrounded exponentials, for the log-sum-exp output.  kMasked: columns >= valid are excluded.
 template <bool kMasked, bool kLse, int kPoly>
@@ -467,27 +464,7 @@ __device__ __forceinline__ void softmax_step(uint32_t tS, uint32_t tP, uint32_t 
   const uint64_t scale2 = pack_f32x2(scale_log2, scale_log2);
   const uint64_t neg_m2 = pack_f32x2(-m_used, -m_used);
   uint64_t sum2 = pack_f32x2(0.f, 0.f), sum_exact2 = pack_f32x2(0.f, 0.f);
-  constexpr int kBlocks = kChunk / 16;   // blocks of 16 columns per trip
-  float e[2][16];                        // exponentials in flight: block b uses e[b & 1]
-  uint32_t pk[8];                        // P of one block (16 columns as bf16 pairs)
-#pragma unroll 1
-  for (int c = 0; c < 128 / kChunk; ++c) {
-#pragma unroll
-    for (int b = 0; b < kBlocks; ++b) {
-      softmax_issue16<kPoly>(s, 16 * b, scale2, neg_m2, e[b & 1]);
-      // round, sum and store the block before this one (the last block of the previous trip when b = 0)
-      if (b > 0 || c > 0) {
-        softmax_finish16<kLse>(e[(b & 1) ^ 1], sum2, sum_exact2, pk);
-        tmem_st8(tP + c * (kChunk / 2) + b * 8 - 8, pk);
-      }
-    }
-    if (kChunk < 128) {
-#pragma unroll
-      for (int i = 0; i < 128 - kChunk; ++i) s[i] = s[i + kChunk];
-    }
-  }
-  softmax_finish16<kLse>(e[1], sum2, sum_exact2, pk);
-  tmem_st8(tP + 56, pk);
+  softmax_row<kLse, kPoly>(s, scale2, neg_m2, sum2, sum_exact2, tP);
 #if AVGGT_PINGPONG
   __syncwarp();
   if (lane == 0) mbar_arrive(smem_u32(&bars->turn[t ^ 1][warp_in_tile]));

@@ -265,12 +265,30 @@ __device__ __forceinline__ uint64_t sub_f32x2(uint64_t a, uint64_t b) {
   asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
-// Volatile form: the compiler keeps these in program order relative to one another, which the
-// softmax loop uses to put its exponentials ahead of the polynomial work of the same block.
+// "_inorder" variants are volatile: the compiler keeps them in program order relative to one
+// another.  AVGGT_INORDER=0 turns them into ordinary instructions (a tuning aid).
+#ifndef AVGGT_INORDER
+#define AVGGT_INORDER 1
+#endif
+#if AVGGT_INORDER
+#define AVGGT_ASM_INORDER asm volatile
+#else
+#define AVGGT_ASM_INORDER asm
+#endif
+__device__ __forceinline__ uint64_t fma_f32x2_inorder(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  AVGGT_ASM_INORDER("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
 __device__ __forceinline__ float ex2_approx_inorder(float x) {
   float y;
-  asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  AVGGT_ASM_INORDER("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2_inorder(float lo, float hi) {
+  uint32_t r;
+  AVGGT_ASM_INORDER("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
 }
 // two floats -> packed bf16x2 (lo in the low half), round to nearest even
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
