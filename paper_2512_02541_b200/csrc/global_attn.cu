@@ -1,21 +1,27 @@
 // Subsampled global attention (Sec. 4.3 of the AVGGT paper) as one fused,
 // warp-specialised flash-style kernel for sm_100a.
 //
-// One CTA owns two tiles of 128 query rows of one head.  Roles:
-//   warps 0-3   softmax of tile 0 (one query row per thread)
-//   warps 4-7   softmax of tile 1
-//   warp  8     TMA producer: Q tiles once, then the compacted K/V of the head
+// One CTA owns two tiles of 128 query rows of one head.  Roles (20 warps):
+//   warps 0-15  softmax.  Warpgroup g = 2 t + h works on query tile t and on
+//               columns [64 h, 64 h + 64) of every 128-key step; within it, warp q
+//               owns rows [32 q, 32 q + 32) (the tensor-memory lanes a warp may
+//               touch), one row per thread.  The two threads that share a row
+//               exchange their half-row maxima through shared memory every step
+//               and their partial sums once at the end.  Four softmax warps per
+//               scheduler keep the exponential unit busy while others wait on
+//               tensor memory, barriers or instruction fetch.
+//   warp  16    TMA producer: Q tiles once, then the compacted K/V of the head
 //               through a ring of shared-memory stages (128-byte swizzle); the
 //               last two ring items are the K/V rows of the CTA's own queries
 //               (the preserved diagonal)
-//   warps 9-10  MMA issuers, one per query tile: S_t = Q_t Kc_j^T and
+//   warps 17-18 MMA issuers, one per query tile: S_t = Q_t Kc_j^T and
 //               O_t += P_t Vc_j with tcgen05.mma, bf16 operands, fp32
 //               accumulators in tensor memory
-//   warp  11    idle (it completes the third warpgroup so that registers can
+//   warp  19    idle (it completes the fifth warpgroup so that registers can
 //               be moved to the softmax warpgroups)
 // Tensor memory per tile: S 128 columns (fp32), P 64 columns (bf16 pairs),
-// O 64 columns (fp32); 512 columns in all.  A softmax thread pulls its row of
-// S into registers and frees S at once, so the next Q K^T runs under the
+// O 64 columns (fp32); 512 columns in all.  A softmax thread pulls its half row
+// of S into registers and frees S at once, so the next Q K^T runs under the
 // exponentials; P V of step j runs under the softmax of step j+1.  The
 // accumulator is rescaled lazily: only when the running maximum grew by more
 // than 2^8 since the last rescale.  The epilogue folds the diagonal and the
@@ -38,10 +44,10 @@ constexpr int kTileKV = 128;     // keys per step
 constexpr int kHeadDim = 64;
 constexpr uint32_t kTileBytes = kTileKV * kHeadDim * 2;   // 16 KiB: one 128 x 64 bf16 tile
 constexpr int kStages = 3;       // K ring and V ring depth
-constexpr int kThreads = 384;
-constexpr int kSoftmaxWarps = 8;
-constexpr int kTmaWarp = 8;
-constexpr int kMmaWarp = 9;
+constexpr int kThreads = 640;
+constexpr int kSoftmaxWarps = 16;
+constexpr int kTmaWarp = 16;
+constexpr int kMmaWarp = 17;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemTileStride = 256;   // columns per query tile: S [0,128) P [128,192) O [192,256)
 constexpr uint32_t kColP = 128, kColO = 192;
@@ -52,19 +58,16 @@ constexpr float kRescaleThreshold = 8.0f;   // log2 units
 // pipe instead of the special-function unit (which, at 16 results per clock per SM, is the
 // scarcest resource of the softmax at head dimension 64).
 #ifndef AVGGT_POLY_EIGHTHS
-#define AVGGT_POLY_EIGHTHS 2
+#define AVGGT_POLY_EIGHTHS 0
 #endif
-// 1: the two softmax warps that share a scheduler (one of each query tile) take turns in the
-// exponential phase, so that one warp's loads, maxima and stores run under the other's exponentials.
+// 1: the softmax warps of the two query tiles that share a scheduler take turns in the
+// exponential phase (two warps at a time saturate the unit), so that one tile's waits, loads,
+// maxima and stores run under the other tile's exponentials instead of all four warps
+// marching in step.
 #ifndef AVGGT_PINGPONG
-#define AVGGT_PINGPONG 0
+#define AVGGT_PINGPONG 1
 #endif
 constexpr int kPolyEighths = AVGGT_POLY_EIGHTHS;
-// How many pairs the rounding and summing of the exponentials trails their issue.
-#ifndef AVGGT_EXP_LAG
-#define AVGGT_EXP_LAG 3
-#endif
-constexpr int kExpLag = AVGGT_EXP_LAG;
 
 struct AttnArgs {
   Plan pl;
@@ -87,7 +90,8 @@ struct __align__(8) Barriers {
   uint64_t s_free[kQTiles];    // softmax -> MMA: S_t(j) has been read into registers
   uint64_t p_full[kQTiles];    // softmax -> MMA: P_t(j) stored (and O_t rescaled)
   uint64_t o_done[kQTiles];    // MMA -> softmax: P_t(j) V_j has completed
-  uint64_t turn[kQTiles][4];   // softmax warp w of the other tile -> warp w of this tile: the exponential unit is yours
+  uint64_t turn[kQTiles][4];   // both warps of rows [32 q, 32 q + 32) of the other tile -> this tile's: the exponential unit is yours
+  uint64_t pair[kQTiles][4];   // the two warps that share rows [32 q, 32 q + 32) of tile t: my half-row value is in shared memory
   uint32_t tmem_base;
   uint32_t abort_flag;
 };
@@ -143,17 +147,18 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 }
 
 // Register budget per thread after the roles have split.  The sum over all warps must not
-// exceed what the launch allocated (168 x 384): a setmaxnreg.inc that asks for more than the
+// exceed what the launch allocated (96 x 640): a setmaxnreg.inc that asks for more than the
 // pool can ever hold waits for ever, and that wait has no time limit.
-constexpr int kRegsSoftmax = 232, kRegsOther = 40;
-static_assert(kRegsSoftmax * kSoftmaxWarps + kRegsOther * (kThreads / 32 - kSoftmaxWarps) <= 168 * (kThreads / 32),
+constexpr int kRegsLaunch = 96;   // 65536 / 640 threads, rounded down to the allocation unit
+constexpr int kRegsSoftmax = 112, kRegsOther = 32;
+static_assert(kRegsSoftmax * kSoftmaxWarps + kRegsOther * (kThreads / 32 - kSoftmaxWarps) <= kRegsLaunch * (kThreads / 32),
               "register budget after setmaxnreg exceeds the launch allocation");
 template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
 // Optional per-phase cycle counters of the softmax loop (a tuning aid; compiled out by default).
 #ifdef AVGGT_PHASE_TIMERS
-__device__ unsigned long long g_phase_cycles[2][4][8];   // [tile][warp of the tile][phase], CTA (0, 0)
+__device__ unsigned long long g_phase_cycles[4][4][8];   // [softmax warpgroup][warp][phase], CTA (0, 0)
 __device__ long long g_trace[64];
 #define AVGGT_TRACE(cond, slot) do { if ((cond) && blockIdx.x == 3 && blockIdx.y == 0) g_trace[slot] = clock64(); } while (0)
 struct PhaseTimers {
@@ -337,91 +342,107 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1
 template <int kPoly>
 __device__ __forceinline__ constexpr bool pair_uses_poly(int g) { return ((g + 1) * kPoly) / 8 != (g * kPoly) / 8; }
 
-// The 128 scores of one query row -> bf16 probabilities, stored to tensor memory at tP as they
-// are produced, relative to the reference maximum folded into neg_m2; adds to the sums for the
-// normaliser (of the rounded values) and for the log-sum-exp (unrounded).
-//
-// A warp issues in order, and an exponential holds the special-function unit for 8 clocks, so
-// the exponentials are spaced out by hand: between two of them sit the scaling of the next pair
-// and the rounding and summing of the pair issued kExpLag pairs earlier (whose results have
-// landed by then).  The "_inorder" instructions are volatile, which keeps them in this order.
+// Values the two threads of a row hand to each other through shared memory.
+struct PairExchange {
+  float step[kQTiles][2][2][kTileQ];    // [tile][step parity][half][row]: half-row maximum of a step
+  float final[kQTiles][2][2][kTileQ];   // [tile][which sum][half][row]: partial sums, once, in the epilogue
+};
+
+// 64 scores of one query row (a half row) -> bf16 probabilities, stored to tensor memory at tP,
+// relative to the reference maximum folded into neg_m2; adds to the sums for the normaliser (of
+// the rounded values) and for the log-sum-exp (unrounded).  Written pair by pair in dependency
+// order; the instruction scheduler interleaves the pairs.
 template <bool kLse, int kPoly>
-__device__ __forceinline__ void softmax_row(const uint32_t (&s)[128], uint64_t scale2, uint64_t neg_m2, uint64_t& sum2,
-                                            uint64_t& sum_exact2, uint32_t tP) {
-  float e0[64], e1[64];   // indexed statically: only the pairs in flight occupy registers
-  uint32_t pk[8];         // P of 16 columns as bf16 pairs
-  uint64_t x2_next = fma_f32x2_inorder(pack_f32x2(__uint_as_float(s[0]), __uint_as_float(s[1])), scale2, neg_m2);
+__device__ __forceinline__ void softmax_half_row(const uint32_t (&s)[64], uint64_t scale2, uint64_t neg_m2, uint64_t& sum2,
+                                                 uint64_t& sum_exact2, uint32_t tP) {
 #pragma unroll
-  for (int i = 0; i < 64 + kExpLag; ++i) {
-    const int k = i - kExpLag;   // the pair that is rounded and summed in this slot
-    float x1 = 0.f;
-    bool mufu = false;
-    if (i < 64) {
-      const uint64_t x2 = x2_next;
-      if (i + 1 < 64)
-        x2_next = fma_f32x2_inorder(pack_f32x2(__uint_as_float(s[2 * i + 2]), __uint_as_float(s[2 * i + 3])), scale2, neg_m2);
-      if (pair_uses_poly<kPoly>(i & 7)) {
-        exp2_poly_pair(x2, e0[i], e1[i]);
+  for (int g = 0; g < 4; ++g) {
+    uint32_t pk[8];   // P of 16 columns as bf16 pairs
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int c = 16 * g + 2 * i;
+      const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), scale2, neg_m2);
+      float p0, p1;
+      if (pair_uses_poly<kPoly>(i)) {
+        exp2_poly_pair(x2, p0, p1);
       } else {
-        float x0;
+        float x0, x1;
         unpack_f32x2(x2, x0, x1);
-        e0[i] = ex2_approx_inorder(x0);
-        mufu = true;
+        p0 = ex2_approx(x0);
+        p1 = ex2_approx(x1);
       }
-    }
-    uint32_t w = 0;
-    if (k >= 0) w = pack_bf16x2_inorder(e0[k], e1[k]);
-    if (mufu) e1[i] = ex2_approx_inorder(x1);
-    if (k >= 0) {
-      pk[k & 7] = w;
-      if (kLse) sum_exact2 = add_f32x2(sum_exact2, pack_f32x2(e0[k], e1[k]));
+      const uint32_t w = pack_bf16x2(p0, p1);
+      pk[i] = w;
+      if (kLse) sum_exact2 = add_f32x2(sum_exact2, pack_f32x2(p0, p1));
       sum2 = add_f32x2(sum2, pack_f32x2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)));
-      if ((k & 7) == 7) tmem_st8(tP + (k >> 3) * 8, pk);
     }
+    tmem_st8(tP + g * 8, pk);
   }
 }
 
-// One step of the online softmax of a query row: S_t(j) in tensor memory -> P_t(j) in tensor
-// memory, running reference maximum and sums updated.
+// What a softmax thread knows about itself.
+struct SoftmaxThread {
+  int t;        // query tile of the CTA
+  int h;        // which half of the 128 columns of a step (and of the 64 output dimensions)
+  int q;        // warp within the warpgroup: rows [32 q, 32 q + 32)
+  int r;        // row within the tile
+  int lane;
+  uint32_t tS, tP, tO;   // tensor-memory addresses of its half of S, P and O (lane included)
+};
+
+// Meeting point of the two warps that share the rows of `me`: returns once both have arrived for
+// the given phase (one phase per step, one more in the epilogue).  What either wrote to shared
+// memory before arriving is visible to the other afterwards.
+__device__ __forceinline__ bool pair_sync(uint32_t phase, const SoftmaxThread& me, Barriers* bars, const AttnArgs& a) {
+  __syncwarp();
+  if (me.lane == 0) mbar_arrive(smem_u32(&bars->pair[me.t][me.q]));
+  return wait_bar(&bars->pair[me.t][me.q], phase & 1, bars, a, 60 + me.t, phase);
+}
+
+// One step of the online softmax of half a query row: S_t(j) in tensor memory -> P_t(j) in
+// tensor memory, running reference maximum and partial sums updated.
 //
-// The row's 128 scores are pulled into registers at once and S_t is released, so that the next
-// Q K^T runs under this step's exponentials.  The row maximum decides whether the reference
-// maximum moves (lazy rescale); then softmax_row takes the exponentials.
+// The half row's 64 scores are pulled into registers at once and the thread's share of S_t is
+// released, so that the next Q K^T runs under this step's exponentials.  The row maximum (of both
+// halves, exchanged with the partner thread) decides whether the reference maximum moves (lazy
+// rescale); both threads of a row take the same decision from the same numbers.
 // kPoly: pairs per eight whose exponential is a polynomial.  kLse: also keep the sum of the
-// unrounded exponentials, for the log-sum-exp output.  kMasked: columns >= valid are excluded.
+// unrounded exponentials, for the log-sum-exp output.  kMasked: columns >= valid are excluded
+// (valid counts from this thread's first column and may be <= 0).
 template <bool kMasked, bool kLse, int kPoly>
-__device__ __forceinline__ void softmax_step(uint32_t tS, uint32_t tP, uint32_t tO, int j, int valid, float scale_log2,
-                                             float& m_used, float& l_run, float& l_exact, Barriers* bars,
-                                             const AttnArgs& a, int t, int warp_in_tile, int lane, bool& ok,
-                                             PhaseTimers& pt) {
-  uint32_t s[128];
+__device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int valid, float scale_log2, float& m_used,
+                                             float& l_run, float& l_exact, Barriers* bars, PairExchange* px,
+                                             const AttnArgs& a, PhaseTimers& pt) {
+  uint32_t s[64];
   {
-    uint32_t (&s4)[4][32] = reinterpret_cast<uint32_t (&)[4][32]>(s);
-    tmem_ld32(tS, s4[0]);
-    tmem_ld32(tS + 32, s4[1]);
-    tmem_ld32(tS + 64, s4[2]);
-    tmem_ld32(tS + 96, s4[3]);
+    uint32_t (&s2)[2][32] = reinterpret_cast<uint32_t (&)[2][32]>(s);
+    tmem_ld32(me.tS, s2[0]);
+    tmem_ld32(me.tS + 32, s2[1]);
   }
   tmem_wait_ld();
   tc_fence_before();
   __syncwarp();
-  if (lane == 0) mbar_arrive(smem_u32(&bars->s_free[t]));
+  if (me.lane == 0) mbar_arrive(smem_u32(&bars->s_free[me.t]));
   pt.lap(1);
-  AVGGT_TRACE(j == 100 && warp_in_tile == 0 && lane == 0, t * 8 + 1);
 
   if (kMasked) {
 #pragma unroll
-    for (int i = 0; i < 128; ++i)
+    for (int i = 0; i < 64; ++i)
       if (i >= valid) s[i] = __float_as_uint(-INFINITY);
   }
-  float mx[4];
+  float mx[2];
 #pragma unroll
-  for (int c = 0; c < 4; ++c) {
+  for (int c = 0; c < 2; ++c) {
     mx[c] = fmaxf(__uint_as_float(s[32 * c]), __uint_as_float(s[32 * c + 1]));
 #pragma unroll
     for (int i = 2; i < 32; i += 2) mx[c] = max3(mx[c], __uint_as_float(s[32 * c + i]), __uint_as_float(s[32 * c + i + 1]));
   }
-  const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;
+  const float half_max = fmaxf(mx[0], mx[1]);
+  // two slots, by step parity: the partner may still be reading the previous step's value
+  px->step[me.t][j & 1][me.h][me.r] = half_max;
+  if (!pair_sync(static_cast<uint32_t>(j), me, bars, a)) return false;
+  const float other_max = *reinterpret_cast<const volatile float*>(&px->step[me.t][j & 1][me.h ^ 1][me.r]);
+  const float tile_max = fmaxf(half_max, other_max) * scale_log2;
   // lazy rescale: keep the old reference maximum unless the new one is far above it
   const bool jump = tile_max > m_used + kRescaleThreshold;
   float alpha = 1.0f;
@@ -433,44 +454,38 @@ __device__ __forceinline__ void softmax_step(uint32_t tS, uint32_t tP, uint32_t 
   }
   const bool rescale = (j > 0) && __any_sync(0xffffffffu, jump);
   pt.lap(2);
-  AVGGT_TRACE(j == 100 && warp_in_tile == 0 && lane == 0, t * 8 + 2);
 
   // P_t(j-1) must have been consumed, and O_t be at rest, before either is written
   if (j > 0) {
-    if (!wait_bar(&bars->o_done[t], (j - 1) & 1, bars, a, 30 + t, j)) { ok = false; return; }
+    if (!wait_bar(&bars->o_done[me.t], (j - 1) & 1, bars, a, 30 + me.t, j)) return false;
     tc_fence_after();
   }
-  if (rescale) {
-#pragma unroll 1
-    for (int h = 0; h < 2; ++h) {
-      uint32_t o[32];
-      tmem_ld32(tO + h * 32, o);
-      tmem_wait_ld();
+  if (rescale) {   // this thread's 32 of the row's 64 accumulator columns
+    uint32_t o[32];
+    tmem_ld32(me.tO, o);
+    tmem_wait_ld();
 #pragma unroll
-      for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-      tmem_st32(tO + h * 32, o);
-    }
+    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+    tmem_st32(me.tO, o);
   }
   pt.lap(3);
 #if AVGGT_PINGPONG
-  // my turn on the exponential unit: the partner warp (same scheduler, other tile) has left its phase
-  if (!wait_bar(&bars->turn[t][warp_in_tile], j & 1, bars, a, 60 + t, j)) { ok = false; return; }
+  // this tile's turn on the exponential unit: the other tile's two warps on this scheduler have left their phase
+  if (!wait_bar(&bars->turn[me.t][me.q], j & 1, bars, a, 62 + me.t, j)) return false;
 #endif
-  pt.lap(4);
-  AVGGT_TRACE(j == 100 && warp_in_tile == 0 && lane == 0, t * 8 + 3);
+  pt.lap(6);
 
   // exponentials, rounded to bf16 for the value product; the normaliser sums the
   // rounded values so that numerator and denominator carry the same weights
   const uint64_t scale2 = pack_f32x2(scale_log2, scale_log2);
   const uint64_t neg_m2 = pack_f32x2(-m_used, -m_used);
   uint64_t sum2 = pack_f32x2(0.f, 0.f), sum_exact2 = pack_f32x2(0.f, 0.f);
-  softmax_row<kLse, kPoly>(s, scale2, neg_m2, sum2, sum_exact2, tP);
+  softmax_half_row<kLse, kPoly>(s, scale2, neg_m2, sum2, sum_exact2, me.tP);
 #if AVGGT_PINGPONG
   __syncwarp();
-  if (lane == 0) mbar_arrive(smem_u32(&bars->turn[t ^ 1][warp_in_tile]));
+  if (me.lane == 0) mbar_arrive(smem_u32(&bars->turn[me.t ^ 1][me.q]));
 #endif
-  pt.lap(5);
-  AVGGT_TRACE(j == 100 && warp_in_tile == 0 && lane == 0, t * 8 + 4);
+  pt.lap(4);
 
   float sum_a, sum_b;
   unpack_f32x2(sum2, sum_a, sum_b);
@@ -482,52 +497,57 @@ __device__ __forceinline__ void softmax_step(uint32_t tS, uint32_t tP, uint32_t 
   tmem_wait_st();
   tc_fence_before();
   __syncwarp();
-  if (lane == 0) mbar_arrive(smem_u32(&bars->p_full[t]));
-  pt.lap(6);
-  AVGGT_TRACE(j == 100 && warp_in_tile == 0 && lane == 0, t * 8 + 6);
+  if (me.lane == 0) mbar_arrive(smem_u32(&bars->p_full[me.t]));
+  pt.lap(5);
+  return true;
 }
 
-__device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, const SmemLayout& sm, uint32_t tmem,
-                                             int t, int wg_tid, int head, int q0) {
+__device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, PairExchange* px, const SmemLayout& sm,
+                                             uint32_t tmem, int warp, int lane, int head, int q0) {
   const Plan& pl = a.pl;
   const int n_kv = a.n_kv_tiles;
-  const int lane = wg_tid & 31;
-  const uint32_t lane_off = static_cast<uint32_t>(wg_tid & ~31) << 16;   // TMEM lane = row within the tile
-  const uint32_t tS = tmem + t * kTmemTileStride + lane_off;
-  const uint32_t tP = tS + kColP, tO = tS + kColO;
-  float m_used = -INFINITY;   // reference maximum of the stored exponentials (log2 units)
-  float l_run = 0.f;          // sum of the bf16-rounded 2^(scale_log2 * s - m_used): normaliser of O
+  SoftmaxThread me;
+  me.t = warp >> 3;
+  me.h = (warp >> 2) & 1;
+  me.q = warp & 3;
+  me.lane = lane;
+  me.r = 32 * me.q + lane;
+  const uint32_t tile_base = tmem + me.t * kTmemTileStride + (static_cast<uint32_t>(32 * me.q) << 16);   // TMEM lane = row
+  me.tS = tile_base + 64 * me.h;
+  me.tP = tile_base + kColP + 32 * me.h;
+  me.tO = tile_base + kColO + 32 * me.h;
+  const int t = me.t, r = me.r;
+  float m_used = -INFINITY;   // reference maximum of the stored exponentials (log2 units); the same in both threads of a row
+  float l_run = 0.f;          // this half's sum of the bf16-rounded 2^(scale_log2 * s - m_used): normaliser of O
   float l_exact = 0.f;        // the same sum without the rounding: log-sum-exp output only
   const bool want_lse = a.lse != nullptr;
-  bool ok = true;
   PhaseTimers pt;
   pt.start();
 #if AVGGT_PINGPONG
   // tile 0 goes first: tile 1 hands it the first turn
-  if (t == 1 && lane == 0) mbar_arrive(smem_u32(&bars->turn[0][wg_tid >> 5]));
+  if (t == 1 && lane == 0) mbar_arrive(smem_u32(&bars->turn[0][me.q]));
 #endif
 
 #pragma unroll 1
-  for (int j = 0; j < n_kv && ok; ++j) {
-    if (!wait_bar(&bars->s_full[t], j & 1, bars, a, 40 + t, j)) { ok = false; break; }
+  for (int j = 0; j < n_kv; ++j) {
+    if (!wait_bar(&bars->s_full[t], j & 1, bars, a, 40 + t, j)) return;
     tc_fence_after();
     pt.lap(0);
-    AVGGT_TRACE(j == 100 && wg_tid == 0, t * 8 + 0);
-    AVGGT_TRACE(j == 101 && wg_tid == 0, t * 8 + 7);
-    const int valid = static_cast<int>(pl.M - static_cast<int64_t>(j) * kTileKV);
+    const int valid_tile = static_cast<int>(pl.M - static_cast<int64_t>(j) * kTileKV);
+    const int valid = valid_tile - 64 * me.h;
+    bool ok;
     // the masked (last, ragged) tile keeps every exponential on the special-function unit, where -inf gives an exact 0
-    if (valid < kTileKV) softmax_step<true, true, 0>(tS, tP, tO, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, a, t, wg_tid >> 5, lane, ok, pt);
-    else if (want_lse) softmax_step<false, true, kPolyEighths>(tS, tP, tO, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, a, t, wg_tid >> 5, lane, ok, pt);
-    else softmax_step<false, false, kPolyEighths>(tS, tP, tO, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, a, t, wg_tid >> 5, lane, ok, pt);
+    if (valid_tile < kTileKV) ok = softmax_step<true, true, 0>(me, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a, pt);
+    else if (want_lse) ok = softmax_step<false, true, kPolyEighths>(me, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a, pt);
+    else ok = softmax_step<false, false, kPolyEighths>(me, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a, pt);
+    if (!ok) return;
   }
-  if (!ok) return;
 #ifdef AVGGT_PHASE_TIMERS
   if (blockIdx.x == 0 && blockIdx.y == 0 && lane == 0)
-    for (int i = 0; i < 8; ++i) g_phase_cycles[t][wg_tid >> 5][i] = pt.acc[i];
+    for (int i = 0; i < 8; ++i) g_phase_cycles[warp >> 2][warp & 3][i] = pt.acc[i];
 #endif
 
-  // ---- epilogue: diagonal and mean-fill terms, normalisation, store
-  const int r = wg_tid;                              // row within the tile
+  // ---- epilogue: diagonal and mean-fill terms, normalisation, store of this thread's 32 output dimensions
   const int row = q0 + t * kTileQ + r;               // query token
   const bool row_valid = row < pl.n_tok;
   bool is_dropped = false;
@@ -535,6 +555,15 @@ __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, 
     const int32_t f = row / pl.L;
     is_dropped = compact_slot(pl, f, row - f * pl.L) < 0;
   }
+  // the row's sums: mine plus the partner's
+  px->final[t][0][me.h][r] = l_run;
+  px->final[t][1][me.h][r] = l_exact;
+  if (!pair_sync(static_cast<uint32_t>(n_kv), me, bars, a)) return;
+  const float other_run = *reinterpret_cast<const volatile float*>(&px->final[t][0][me.h ^ 1][r]);
+  const float other_exact = *reinterpret_cast<const volatile float*>(&px->final[t][1][me.h ^ 1][r]);
+  l_run += other_run;
+  l_exact += other_exact;
+
   if (!wait_bar(&bars->o_done[t], (n_kv - 1) & 1, bars, a, 50 + t, n_kv)) return;
   tc_fence_after();
   if (!wait_bar(&bars->q_full, 0, bars, a, 52, 0)) return;   // completed long ago: makes the Q tile visible to this thread
@@ -547,7 +576,8 @@ __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, 
     if (!wait_bar(&bars->v_full[item % kStages], par, bars, a, 54, item)) return;
   }
   const uint8_t* sQ = sm.q[t];
-  float l_d = -INFINITY, l_m = -INFINITY;            // base-2 logits of the two extra columns
+  // base-2 logits of the two extra columns; both threads of a row compute them in full, from the same numbers
+  float l_d = -INFINITY, l_m = -INFINITY;
   if (a.use_diag && is_dropped) {
     float acc = 0.f;
 #pragma unroll
@@ -583,20 +613,19 @@ __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, 
   const float inv_z = 1.0f / z;
   const float w_s = a_s * inv_z, w_d = p_d * inv_z, w_m = p_m * inv_z;
 
-  uint32_t o[2][32];
-  tmem_ld32(tO, o[0]);
-  tmem_ld32(tO + 32, o[1]);
+  uint32_t o[32];
+  tmem_ld32(me.tO, o);
   tmem_wait_ld();
   if (row_valid) {
-    uint4* dst = reinterpret_cast<uint4*>(a.O + (static_cast<size_t>(row) * pl.H + head) * kHeadDim);
-    const float4* vm = reinterpret_cast<const float4*>(a.vmean + head * kHeadDim);
+    uint4* dst = reinterpret_cast<uint4*>(a.O + (static_cast<size_t>(row) * pl.H + head) * kHeadDim) + 4 * me.h;
+    const float4* vm = reinterpret_cast<const float4*>(a.vmean + head * kHeadDim) + 8 * me.h;
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
+    for (int c = 0; c < 4; ++c) {
       float v[8];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(o[c >> 2][(c & 3) * 8 + e]) * w_s;
+      for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(o[c * 8 + e]) * w_s;
       if (w_d != 0.f) {
-        const uint4 vd = ld_swizzled(sVd, r, c);
+        const uint4 vd = ld_swizzled(sVd, r, 4 * me.h + c);
         const uint32_t w[4] = {vd.x, vd.y, vd.z, vd.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -616,7 +645,7 @@ __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, 
       out.w = pack_bf16x2(v[6], v[7]);
       dst[c] = out;
     }
-    if (want_lse) {
+    if (want_lse && me.h == 0) {
       const float z_exact = fmaf(l_exact, a_s, p_d + p_m);
       a.lse[static_cast<size_t>(row) * pl.H + head] = (m_fin + log2f(z_exact)) * 0.6931471805599453f;
     }
@@ -635,6 +664,7 @@ global_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   sm.k = smem + kQTiles * kTileBytes;
   sm.v = sm.k + kStages * kTileBytes;
   __shared__ Barriers bars;
+  __shared__ PairExchange pair_exchange;
 
   const int tid = threadIdx.x;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // warp-uniform by construction
@@ -654,10 +684,11 @@ global_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     }
     for (int t = 0; t < kQTiles; ++t) {
       mbar_init(smem_u32(&bars.s_full[t]), 1);
-      mbar_init(smem_u32(&bars.s_free[t]), 4);
-      mbar_init(smem_u32(&bars.p_full[t]), 4);
+      mbar_init(smem_u32(&bars.s_free[t]), kSoftmaxWarps / kQTiles);
+      mbar_init(smem_u32(&bars.p_full[t]), kSoftmaxWarps / kQTiles);
       mbar_init(smem_u32(&bars.o_done[t]), 1);
-      for (int w = 0; w < 4; ++w) mbar_init(smem_u32(&bars.turn[t][w]), 1);
+      for (int w = 0; w < 4; ++w) mbar_init(smem_u32(&bars.pair[t][w]), 2);
+      for (int w = 0; w < 4; ++w) mbar_init(smem_u32(&bars.turn[t][w]), 2);
     }
     bars.abort_flag = 0;
     fence_mbar_init();
@@ -673,8 +704,7 @@ global_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
   if (warp < kSoftmaxWarps) {
     reg_inc<kRegsSoftmax>();
-    const int t = warp >> 2;
-    softmax_role(a, &bars, sm, tmem, t, tid & 127, head, q0);
+    softmax_role(a, &bars, &pair_exchange, sm, tmem, warp, tid & 31, head, q0);
   } else {
     reg_dec<kRegsOther>();
     if (warp == kTmaWarp) producer_role(&tm_q, &tm_k, &tm_v, &tm_kc, &tm_vc, a, &bars, sm, head, q0);
@@ -694,7 +724,7 @@ constexpr size_t kAttnSmemBytes = static_cast<size_t>(kTileBytes) * (kQTiles + 2
 size_t global_attn_ws_bytes(const Plan&, int) { return kAttnStatusBytes; }
 
 #ifdef AVGGT_PHASE_TIMERS
-// Tuning aids: copy the 2 x 4 x 8 phase counters / the 64 event stamps of the last launch to the host.
+// Tuning aids: copy the 4 x 4 x 8 phase counters / the 64 event stamps of the last launch to the host.
 extern "C" int avggt_debug_phase_cycles(unsigned long long* out64) {
   return cudaMemcpyFromSymbol(out64, g_phase_cycles, sizeof(g_phase_cycles)) == cudaSuccess ? 0 : -1;
 }
