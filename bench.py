@@ -33,9 +33,13 @@ if ROOT not in sys.path:
 from paper_2512_02541_b200 import inputs  # noqa: E402
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
-# profiles/ (global_attn_kernel_*, build_kv_kernel_*); None where no capture of that workload exists.
+# profiles/; None where no capture covers the workload.  The attention kernel is captured on the 30-frame copy of
+# the layer (profiles/global_attn_kernel_vggt_n30_s4.md); its traffic is proportional to the frame count, so the
+# 100-frame figure is that capture x 100/30.  The compaction kernel is captured on the 100-frame workload itself.
+_ATTN_N30 = 0.299476e9 + 0.071481e9
 NCU_TRAFFIC = {
-    "vggt_n100_s4": {"global_attn_kernel": 1.355360e9 + 0.268312e9, "build_kv_kernel": 0.562812e9 + 0.104510e9},
+    "vggt_n30_s4": {"global_attn_kernel": _ATTN_N30},
+    "vggt_n100_s4": {"global_attn_kernel": _ATTN_N30 * 100 / 30, "build_kv_kernel": 0.562812e9 + 0.104510e9},
 }
 
 METRIC = "subsampled_global_attn_queries_per_sec"
