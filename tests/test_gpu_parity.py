@@ -153,6 +153,26 @@ def test_vggt_100_frames_sampled_rows():
     assert torch.isfinite(O.float()).all()
 
 
+@pytest.mark.parametrize("name,n_rows", [
+    ("vggt_n300_s6", 96),     # 412,200 queries x 75,600 compact keys
+    ("vggt_n800_s9", 64),     # 1,099,200 queries x 139,200 compact keys: the long-context case
+    ("vggt_n333_s1", 48),     # dense layer (both switches off), 457,542 x 457,542
+    ("vggt_n333_s9", 64),     # the other end of the factor sweep
+])
+def test_full_size_configs_sampled_rows(name, n_rows):
+    """The larger benchmark configurations at full size, in the launch configuration bench.py times:
+    compaction checked in full against the oracle, attention on a stratified sample of rows the
+    oracle computes one by one, and every output row finite."""
+    wl = inputs.WORKLOADS[name]
+    params, ocfg, layer, Q, K, V, O = _run_gpu(wl)
+    Kh, Vh = _check_build(ocfg, layer, K, V)
+    rows = inputs.sample_rows(wl, n_rows).numpy()
+    _check_attn(ocfg, Q, Kh, Vh, O, rows=rows)
+    assert torch.isfinite(O.float()).all()
+    del Q, K, V, O, layer
+    torch.cuda.empty_cache()
+
+
 def test_results_are_deterministic():
     wl = inputs.Workload("det", 5, 16, 16, 5, 4, 64, 4, 1, 2, "iid")
     params, _ = _cfgs(wl)
