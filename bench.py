@@ -167,6 +167,22 @@ class ClockSampler:
         return out
 
 
+def max_over_ranks(values, device, world):
+    """Every rank passes its own device-timed durations; all get the element-wise maximum over the ranks
+    (the replicas of a multi-GPU run are timed by the slowest one).  One rank: the values themselves."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_throughput(units_per_rank, world, ms_per_step):
+    """Aggregate metric of N replicas: the units all ranks processed per second of the slowest rank's step."""
+    return world * units_per_rank / (ms_per_step * 1e-3)
+
+
 def run_ours(args, wl):
     import torch.distributed as dist
 
@@ -239,15 +255,12 @@ def run_ours(args, wl):
     barrier()
     e2e_ms = s0.elapsed_time(s1)
 
-    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = times.tolist()
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dev if world > 1 else "cpu", world)
 
     if rank == 0:
         peaks = _peaks()
         ms_per_step = total_ms / args.steps
-        value = world * n_q / (ms_per_step * 1e-3)
+        value = whole_job_throughput(n_q, world, ms_per_step)
         flops = 4.0 * n_q * M * H * d
         attn_avg = sum(attn_ms) / len(attn_ms)
         build_avg = sum(build_ms) / len(build_ms)
