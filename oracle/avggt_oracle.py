@@ -284,3 +284,37 @@ def global_attn_blocked(cfg, Q, K, V, rows, return_lse=False):
         O[:, h, :] = o / z[:, None]
         lse[:, h] = mx + np.log(z)
     return (O, lse) if return_lse else O
+
+
+def frame_attn(cfg, Q, K, V, rows=None, return_lse=False):
+    """Frame attention of a converted early global block (Sec. 4.2, "Global-to-Frame Attention
+    Conversion"): the (B, N L, C) rearrangement is skipped, so every token attends to the L tokens
+    of its own frame only (special tokens included), with plain softmax attention.  Nothing is
+    subsampled; sigma, diag and mean_fill of ``cfg`` play no part.
+
+    Q, K, V: [N*L, H, d].  Returns O [len(rows), H, d] float64 (and the natural-log normaliser
+    [len(rows), H] with ``return_lse``) for the query rows ``rows`` (default: all), one row at a
+    time: logits over the frame's keys, one softmax, weighted sum of the frame's values.
+    """
+    Q, K, V = np.asarray(Q), np.asarray(K), np.asarray(V)
+    H, d, L = cfg.n_heads, cfg.head_dim, cfg.tokens_per_frame
+    assert Q.shape == (cfg.n_tokens, H, d) and K.shape == Q.shape and V.shape == Q.shape
+    scale = cfg.scale
+    if rows is None:
+        rows = np.arange(cfg.n_tokens)
+    rows = np.asarray(rows, dtype=np.int64)
+    O = np.empty((len(rows), H, d), dtype=np.float64)
+    lse = np.empty((len(rows), H), dtype=np.float64)
+    for out_i, i in enumerate(rows):
+        f = int(i) // L                                   # the query's frame
+        Kf = K[f * L:(f + 1) * L].astype(np.float64)      # [L, H, d]
+        Vf = V[f * L:(f + 1) * L].astype(np.float64)
+        q = Q[i].astype(np.float64)                       # [H, d]
+        logits = scale * np.einsum("hd,lhd->hl", q, Kf)   # [H, L]
+        mx = logits.max(axis=1, keepdims=True)
+        p = np.exp(logits - mx)
+        z = p.sum(axis=1, keepdims=True)
+        O[out_i] = np.einsum("hl,lhd->hd", p / z, Vf)
+        lse[out_i] = (mx + np.log(z))[:, 0]
+    return (O, lse) if return_lse else O
+

@@ -323,3 +323,54 @@ def test_lse_is_log_of_summed_exponentials():
             tot = sum(math.exp(scale * float(Q[i, h] @ K[j, h])) for j in range(cfg.n_tokens) if not D[j] or j == i)
             tot += (int(D.sum()) - int(D[i])) * math.exp(scale * float(Q[i, h] @ kbar))
             assert abs(lse[i, h] - math.log(tot)) < 1e-12
+
+
+# --------------------------------------------------------------------------
+# frame attention of converted early global blocks (Sec. 4.2)
+# --------------------------------------------------------------------------
+
+def test_frame_attn_is_per_frame_library_sdpa():
+    """Skipping the (B, N L, C) rearrangement means N independent dense attentions: each frame
+    against a library routine, in the (B N, L, C) layout the paper names."""
+    cfg = orc.SGAConfig(4, 3, 5, 2, 3, 16, sigma=4)
+    Q, K, V = _rand_qkv(cfg, seed=21)
+    L, H, d = cfg.tokens_per_frame, cfg.n_heads, cfg.head_dim
+    tq, tk, tv = (torch.from_numpy(a).reshape(cfg.n_frames, L, H, d).permute(0, 2, 1, 3) for a in (Q, K, V))   # [N,H,L,d]
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv).permute(0, 2, 1, 3).reshape(-1, H, d).numpy()
+    got, lse = orc.frame_attn(cfg, Q, K, V, return_lse=True)
+    np.testing.assert_allclose(got, ref, rtol=0, atol=1e-12)
+    # the normaliser against its definition, frame by frame
+    logits = np.einsum("nlhd,nmhd->nhlm", Q.reshape(cfg.n_frames, L, H, d), K.reshape(cfg.n_frames, L, H, d)) / math.sqrt(d)
+    want_lse = np.log(np.exp(logits).sum(axis=-1)).transpose(0, 2, 1).reshape(-1, H)
+    np.testing.assert_allclose(lse, want_lse, rtol=0, atol=1e-12)
+
+
+def test_frame_attn_equals_one_frame_global_attention():
+    """With a single frame, global and frame attention are the same layer (the O((N L)^2) -> O(N L^2)
+    statement at N = 1), and other frames' tokens cannot influence a frame's output."""
+    cfg = orc.SGAConfig(3, 4, 4, 5, 2, 8, sigma=2)
+    Q, K, V = _rand_qkv(cfg, seed=22)
+    L = cfg.tokens_per_frame
+    one = orc.SGAConfig(1, 4, 4, 5, 2, 8, sigma=1, diag=False, mean_fill=0)
+    got = orc.frame_attn(cfg, Q, K, V)
+    for f in range(cfg.n_frames):
+        sl = slice(f * L, (f + 1) * L)
+        np.testing.assert_allclose(got[sl], orc.global_attn(one, Q[sl], K[sl], V[sl]), rtol=0, atol=1e-12)
+    K2, V2 = K.copy(), V.copy()
+    K2[L:2 * L] += 5.0                       # disturb frame 1 only
+    V2[L:2 * L] -= 3.0
+    got2 = orc.frame_attn(cfg, Q, K2, V2)
+    np.testing.assert_array_equal(got2[:L], got[:L])
+    np.testing.assert_array_equal(got2[2 * L:], got[2 * L:])
+    assert np.abs(got2[L:2 * L] - got[L:2 * L]).max() > 1e-3
+
+
+def test_frame_attn_rows_and_switches():
+    """A subset of rows gives the same rows; sigma, diag and mean_fill play no part."""
+    a = orc.SGAConfig(3, 3, 4, 1, 2, 8, sigma=9, diag=True, mean_fill=2)
+    b = orc.SGAConfig(3, 3, 4, 1, 2, 8, sigma=1, diag=False, mean_fill=0)
+    Q, K, V = _rand_qkv(a, seed=23)
+    full = orc.frame_attn(a, Q, K, V)
+    rows = np.array([0, 12, 13, 25, 38])
+    np.testing.assert_array_equal(orc.frame_attn(a, Q, K, V, rows=rows), full[rows])
+    np.testing.assert_array_equal(orc.frame_attn(b, Q, K, V), full)
