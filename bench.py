@@ -234,6 +234,18 @@ def run_ours(args, wl):
     build_ms = [e[0].elapsed_time(e[1]) for e in ev]
     attn_ms = [e[1].elapsed_time(e[2]) for e in ev]
 
+    # ---- outside the timed region: the same tokens through frame attention (Sec. 4.2), for the report
+    fe = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    layer.frame_attend(Q, K, V, out=O)
+    barrier()
+    fe[0].record(stream)
+    for _ in range(args.steps):
+        layer.frame_attend(Q, K, V, out=O)
+    fe[1].record(stream)
+    barrier()
+    layer.check_status()
+    frame_ms = fe[0].elapsed_time(fe[1]) / args.steps
+
     # ---- end to end through the public API with host buffers
     e2e_steps = max(1, min(args.steps, 5))
     hQ, hK, hV = (t.cpu().pin_memory() for t in (Q, K, V))
@@ -282,6 +294,8 @@ def run_ours(args, wl):
             "tflops": world * flops / (ms_per_step * 1e-3) / 1e12,
             "attn_ms": attn_avg, "attn_ms_min": min(attn_ms), "build_kv_ms": build_avg, "build_kv_ms_min": min(build_ms),
             "attn_queries_per_sec": n_q / (attn_avg * 1e-3),
+            "frame_attn_ms": frame_ms,
+            "frame_attn_tflops": 4.0 * n_q * wl.tokens_per_frame * H * d / (frame_ms * 1e-3) / 1e12,
             "roofline": {"bound": "tensor", "kernel": "global_attn_kernel", "achieved": achieved_tf, "peak": peak_tf,
                          "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
                          "traffic": NCU_TRAFFIC.get(wl.name, {}).get("global_attn_kernel"),

@@ -171,6 +171,26 @@ int avggt_global_attn(const avggt_params* p, const void* Q, const void* K, const
                       void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Frame attention of a converted early global block (Sec. 4.2, "Global-to-Frame Attention
+ * Conversion"): the (B, N L, C) rearrangement is skipped, so every token attends to the L tokens
+ * of its own frame only, special tokens included, with plain softmax attention:
+ *   O[i][h][:] = sum_{j in frame(i)} softmax_j(scale q_i.k_j) V[j][h][:].
+ * N independent dense problems in one launch of the same kernel; keys and values are read
+ * straight from K and V (nothing is compacted), so avggt_build_kv is not needed.  Of `p` the
+ * call uses n_frames, tokens_per_frame, n_heads, head_dim and softmax_scale; sigma, diag,
+ * mean_fill and flags play no part but must be valid.  n_frames <= 65535.
+ *
+ *   Q, K, V       device, bf16 [N*L, H, d]; must be finite (a tile of keys may reach into the
+ *                 next frame's rows, whose products are masked to zero weight)
+ *   O             device, bf16 [N*L, H, d]       written
+ *   lse           device, float [N*L, H] or NULL
+ *   ws            device scratch of at least attn_ws_bytes (avggt_workspace_bytes); status
+ *                 block as for avggt_global_attn
+ */
+int avggt_frame_attn(const avggt_params* p, const void* Q, const void* K, const void* V,
+                     void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * After the caller has synchronised the stream: reads the status block at the start of an
  * attention workspace (a 16-byte device-to-host copy) and returns AVGGT_OK or
  * AVGGT_ERR_DEVICE_TIMEOUT if a bounded wait inside the kernel gave up (the output is then

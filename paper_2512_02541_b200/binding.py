@@ -25,6 +25,7 @@ AVGGT_MEAN_OFF, AVGGT_MEAN_UNIT, AVGGT_MEAN_FILL = 0, 1, 2
 # every symbol include/avggt.h declares
 EXPORTS = (
     "avggt_kv_count", "avggt_workspace_bytes", "avggt_build_kv", "avggt_build_kv_noalloc", "avggt_global_attn",
+    "avggt_frame_attn",
     "avggt_check_status", "avggt_strerror", "avggt_last_cuda_error", "avggt_version",
 )
 
@@ -82,6 +83,8 @@ def lib():
         L.avggt_build_kv_noalloc.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.avggt_build_kv_noalloc.restype = ctypes.c_int
         L.avggt_global_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.avggt_frame_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.avggt_frame_attn.restype = ctypes.c_int
         L.avggt_check_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
         L.avggt_strerror.argtypes = [ctypes.c_int]
         for f in (L.avggt_kv_count, L.avggt_workspace_bytes, L.avggt_build_kv, L.avggt_global_attn, L.avggt_check_status):
@@ -147,6 +150,12 @@ def avggt_global_attn(params, Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws, ws_byte
     """Enqueue the subsampled global attention."""
     _check(lib().avggt_global_attn(ctypes.byref(params), _ptr(Q), _ptr(K), _ptr(V), _ptr(Kc), _ptr(Vc), _ptr(kmean),
                                    _ptr(vmean), _ptr(O), _ptr(lse), _ptr(ws), ws_bytes, stream), "avggt_global_attn")
+
+
+def avggt_frame_attn(params, Q, K, V, O, lse, ws, ws_bytes, stream=None):
+    """Enqueue the frame attention of a converted early global block (every frame on its own)."""
+    _check(lib().avggt_frame_attn(ctypes.byref(params), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(lse), _ptr(ws),
+                                  ws_bytes, stream), "avggt_frame_attn")
 
 
 def avggt_check_status(attn_ws):

@@ -169,6 +169,29 @@ int avggt_global_attn(const avggt_params* p, const void* Q, const void* K, const
   return record_cuda(e);
 }
 
+int avggt_frame_attn(const avggt_params* p, const void* Q, const void* K, const void* V, void* O, float* lse, void* ws,
+                     size_t ws_bytes, void* cuda_stream) {
+  Plan pl;
+  int rc = make_plan(p, &pl);
+  if (rc != AVGGT_OK) return rc;
+  if (!Q || !K || !V || !O || !ws) return AVGGT_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(ws) ||
+      (reinterpret_cast<uintptr_t>(lse) & 3u))
+    return AVGGT_ERR_ALIGNMENT;
+  if (pl.n_frames > 65535) return AVGGT_ERR_UNSUPPORTED;
+  DeviceInfo di;
+  rc = device_info(&di);
+  if (rc != AVGGT_OK) return rc;
+  if (ws_bytes < global_attn_ws_bytes(pl, di.sm_count)) return AVGGT_ERR_WORKSPACE_TOO_SMALL;
+  bool tmap_failed = false;
+  cudaError_t e = launch_frame_attn(pl, Q, K, V, O, lse, ws, static_cast<cudaStream_t>(cuda_stream), &tmap_failed);
+  if (tmap_failed) {
+    std::strncpy(g_cuda_error, "cuTensorMapEncodeTiled failed", sizeof(g_cuda_error) - 1);
+    return AVGGT_ERR_CUDA;
+  }
+  return record_cuda(e);
+}
+
 int avggt_check_status(const void* attn_ws, uint32_t* detail) {
   if (!attn_ws) return AVGGT_ERR_INVALID_ARG;
   uint32_t st[4] = {0, 0, 0, 0};

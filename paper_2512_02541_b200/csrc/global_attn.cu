@@ -76,7 +76,10 @@ struct AttnArgs {
   __nv_bfloat16* O;     // [n_tok, H, d]
   float* lse;           // [n_tok, H] or null
   uint32_t* status;     // 4 words
-  int32_t n_kv_tiles;   // ceil(M / 128)
+  int32_t frame_mode;   // 0: subsampled global attention over the compact keys.  1: frame attention (Sec. 4.2):
+                        //    blockIdx.z is the frame, keys and values are the frame's own rows of K and V
+  int64_t n_keys;       // keys of one problem: M, or the tokens of a frame
+  int32_t n_kv_tiles;   // ceil(n_keys / 128)
   int32_t use_diag;     // diag on and |D| > 0
   int32_t use_mean;     // mean_fill on and |D| > 0
   float scale_log2;     // softmax scale * log2(e)
@@ -98,7 +101,7 @@ struct __align__(8) Barriers {
 
 __device__ __forceinline__ void report_timeout(const AttnArgs& a, Barriers* bars, uint32_t where, uint32_t iter) {
   if (atomicCAS(a.status, 0u, 1u) == 0u) {
-    a.status[1] = blockIdx.x + blockIdx.y * gridDim.x;
+    a.status[1] = blockIdx.x + (blockIdx.y + blockIdx.z * gridDim.y) * gridDim.x;
     a.status[2] = where;
     a.status[3] = iter;
   }
@@ -175,6 +178,14 @@ struct PhaseTimers {
 };
 #endif
 
+// What one CTA works on.
+struct CtaProblem {
+  int head;
+  int q0;             // first query row (token index) of the CTA's two tiles
+  int64_t row_end;    // query rows at or beyond this token index are not stored
+  int key_row0;       // frame attention: token index of the frame's first key
+};
+
 struct SmemLayout {
   uint8_t* q[kQTiles];
   uint8_t* k;   // kStages tiles
@@ -195,9 +206,10 @@ __device__ __forceinline__ bool wait_bar_warp(uint64_t* bar, uint32_t parity, Ba
 // ------------------------------------------------------------------ TMA producer (one warp)
 __device__ __forceinline__ void producer_role(const CUtensorMap* tm_q, const CUtensorMap* tm_k, const CUtensorMap* tm_v,
                                               const CUtensorMap* tm_kc, const CUtensorMap* tm_vc, const AttnArgs& a,
-                                              Barriers* bars, const SmemLayout& sm, int head, int q0) {
+                                              Barriers* bars, const SmemLayout& sm, const CtaProblem& cta) {
   const int n_kv = a.n_kv_tiles;
   const int n_items = n_kv + (a.use_diag ? kQTiles : 0);
+  const int head = cta.head, q0 = cta.q0;
   if (elect_one()) {
     prefetch_tensormap(tm_q);
     prefetch_tensormap(tm_kc);
@@ -218,7 +230,8 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tm_q, const CUt
     if (elect_one()) {
       const uint32_t kb = smem_u32(&bars->k_full[stage]);
       mbar_arrive_expect_tx(kb, kTileBytes);
-      if (it < n_kv) tma_load_3d(smem_u32(sm.k + stage * kTileBytes), tm_kc, 0, it * kTileKV, head, kb);
+      if (a.frame_mode) tma_load_2d(smem_u32(sm.k + stage * kTileBytes), tm_k, head * kHeadDim, cta.key_row0 + it * kTileKV, kb);
+      else if (it < n_kv) tma_load_3d(smem_u32(sm.k + stage * kTileBytes), tm_kc, 0, it * kTileKV, head, kb);
       else tma_load_2d(smem_u32(sm.k + stage * kTileBytes), tm_k, head * kHeadDim, q0 + (it - n_kv) * kTileQ, kb);
     }
     __syncwarp();
@@ -227,7 +240,8 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tm_q, const CUt
     if (elect_one()) {
       const uint32_t vb = smem_u32(&bars->v_full[stage]);
       mbar_arrive_expect_tx(vb, kTileBytes);
-      if (it < n_kv) tma_load_3d(smem_u32(sm.v + stage * kTileBytes), tm_vc, 0, it * kTileKV, head, vb);
+      if (a.frame_mode) tma_load_2d(smem_u32(sm.v + stage * kTileBytes), tm_v, head * kHeadDim, cta.key_row0 + it * kTileKV, vb);
+      else if (it < n_kv) tma_load_3d(smem_u32(sm.v + stage * kTileBytes), tm_vc, 0, it * kTileKV, head, vb);
       else tma_load_2d(smem_u32(sm.v + stage * kTileBytes), tm_v, head * kHeadDim, q0 + (it - n_kv) * kTileQ, vb);
     }
     __syncwarp();
@@ -503,7 +517,7 @@ __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int
 }
 
 __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, PairExchange* px, const SmemLayout& sm,
-                                             uint32_t tmem, int warp, int lane, int head, int q0) {
+                                             uint32_t tmem, int warp, int lane, const CtaProblem& cta) {
   const Plan& pl = a.pl;
   const int n_kv = a.n_kv_tiles;
   SoftmaxThread me;
@@ -533,7 +547,7 @@ __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, 
     if (!wait_bar(&bars->s_full[t], j & 1, bars, a, 40 + t, j)) return;
     tc_fence_after();
     pt.lap(0);
-    const int valid_tile = static_cast<int>(pl.M - static_cast<int64_t>(j) * kTileKV);
+    const int valid_tile = static_cast<int>(a.n_keys - static_cast<int64_t>(j) * kTileKV);
     const int valid = valid_tile - 64 * me.h;
     bool ok;
     // the masked (last, ragged) tile keeps every exponential on the special-function unit, where -inf gives an exact 0
@@ -548,8 +562,9 @@ __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, 
 #endif
 
   // ---- epilogue: diagonal and mean-fill terms, normalisation, store of this thread's 32 output dimensions
-  const int row = q0 + t * kTileQ + r;               // query token
-  const bool row_valid = row < pl.n_tok;
+  const int head = cta.head;
+  const int row = cta.q0 + t * kTileQ + r;           // query token
+  const bool row_valid = row < cta.row_end;
   bool is_dropped = false;
   if (row_valid && pl.n_dropped > 0) {
     const int32_t f = row / pl.L;
@@ -668,8 +683,17 @@ global_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
   const int tid = threadIdx.x;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // warp-uniform by construction
-  const int head = blockIdx.y;
-  const int q0 = blockIdx.x * (kQTiles * kTileQ);
+  CtaProblem cta;
+  cta.head = blockIdx.y;
+  if (a.frame_mode) {
+    cta.key_row0 = static_cast<int>(blockIdx.z) * a.pl.L;
+    cta.q0 = cta.key_row0 + blockIdx.x * (kQTiles * kTileQ);
+    cta.row_end = static_cast<int64_t>(cta.key_row0) + a.pl.L;
+  } else {
+    cta.key_row0 = 0;
+    cta.q0 = blockIdx.x * (kQTiles * kTileQ);
+    cta.row_end = a.pl.n_tok;
+  }
 
   // a launch in which a wait has already run out is abandoned: the remaining CTAs leave at once
   if (__syncthreads_or(*reinterpret_cast<volatile uint32_t*>(a.status) != 0u)) return;
@@ -704,10 +728,10 @@ global_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
   if (warp < kSoftmaxWarps) {
     reg_inc<kRegsSoftmax>();
-    softmax_role(a, &bars, &pair_exchange, sm, tmem, warp, tid & 31, head, q0);
+    softmax_role(a, &bars, &pair_exchange, sm, tmem, warp, tid & 31, cta);
   } else {
     reg_dec<kRegsOther>();
-    if (warp == kTmaWarp) producer_role(&tm_q, &tm_k, &tm_v, &tm_kc, &tm_vc, a, &bars, sm, head, q0);
+    if (warp == kTmaWarp) producer_role(&tm_q, &tm_k, &tm_v, &tm_kc, &tm_vc, a, &bars, sm, cta);
     else if (warp == kMmaWarp) mma_role<0>(a, &bars, sm, tmem);
     else if (warp == kMmaWarp + 1) mma_role<1>(a, &bars, sm, tmem);
   }
@@ -733,9 +757,12 @@ extern "C" int avggt_debug_trace(long long* out64) {
 }
 #endif
 
-cudaError_t launch_global_attn(const Plan& pl, int /*sm_count*/, const void* Q, const void* K, const void* V,
-                               const void* Kc, const void* Vc, const float* kmean, const float* vmean, void* O,
-                               float* lse, void* ws, cudaStream_t st, bool* tmap_failed) {
+namespace {
+
+// Tensor maps and launch shared by the two entry points.  frame_mode: see AttnArgs.
+cudaError_t launch_attn(const Plan& pl, bool frame_mode, const void* Q, const void* K, const void* V, const void* Kc,
+                        const void* Vc, const float* kmean, const float* vmean, void* O, float* lse, void* ws,
+                        cudaStream_t st, bool* tmap_failed) {
   *tmap_failed = false;
   AttnArgs a;
   a.pl = pl;
@@ -744,24 +771,33 @@ cudaError_t launch_global_attn(const Plan& pl, int /*sm_count*/, const void* Q, 
   a.O = static_cast<__nv_bfloat16*>(O);
   a.lse = lse;
   a.status = static_cast<uint32_t*>(ws);
-  a.n_kv_tiles = static_cast<int32_t>((pl.M + kTileKV - 1) / kTileKV);
-  a.use_diag = (pl.diag != 0 && pl.n_dropped > 0) ? 1 : 0;
-  a.use_mean = (pl.mean_fill != 0 && pl.n_dropped > 0) ? 1 : 0;
+  a.frame_mode = frame_mode ? 1 : 0;
+  a.n_keys = frame_mode ? pl.L : pl.M;
+  a.n_kv_tiles = static_cast<int32_t>((a.n_keys + kTileKV - 1) / kTileKV);
+  a.use_diag = (!frame_mode && pl.diag != 0 && pl.n_dropped > 0) ? 1 : 0;
+  a.use_mean = (!frame_mode && pl.mean_fill != 0 && pl.n_dropped > 0) ? 1 : 0;
   a.scale_log2 = pl.scale * kLog2e;
 
-  // token-major [n_tok, H*d] maps for Q and (diagonal tiles) K, V; head-major [H, M, d] maps for Kc, Vc
+  // token-major [n_tok, H*d] maps for Q and for K, V (the diagonal tiles; all tiles of frame attention);
+  // head-major [H, M, d] maps for Kc, Vc
   CUtensorMap tm_q, tm_k, tm_v, tm_kc, tm_vc;
   const uint64_t tok_dims[2] = {static_cast<uint64_t>(pl.H) * pl.d, static_cast<uint64_t>(pl.n_tok)};
   const uint64_t tok_str[1] = {static_cast<uint64_t>(pl.H) * pl.d * 2};
   const uint32_t tok_box[2] = {kHeadDim, kTileQ};
-  const uint64_t c_dims[3] = {static_cast<uint64_t>(pl.d), static_cast<uint64_t>(pl.M), static_cast<uint64_t>(pl.H)};
-  const uint64_t c_str[2] = {static_cast<uint64_t>(pl.d) * 2, static_cast<uint64_t>(pl.M) * pl.d * 2};
-  const uint32_t c_box[3] = {kHeadDim, kTileKV, 1};
+  const bool reads_kv = frame_mode || a.use_diag;
   bool good = make_tmap_bf16(&tm_q, Q, 2, tok_dims, tok_str, tok_box);
-  good = good && make_tmap_bf16(&tm_k, a.use_diag ? K : Q, 2, tok_dims, tok_str, tok_box);
-  good = good && make_tmap_bf16(&tm_v, a.use_diag ? V : Q, 2, tok_dims, tok_str, tok_box);
-  good = good && make_tmap_bf16(&tm_kc, Kc, 3, c_dims, c_str, c_box);
-  good = good && make_tmap_bf16(&tm_vc, Vc, 3, c_dims, c_str, c_box);
+  good = good && make_tmap_bf16(&tm_k, reads_kv ? K : Q, 2, tok_dims, tok_str, tok_box);
+  good = good && make_tmap_bf16(&tm_v, reads_kv ? V : Q, 2, tok_dims, tok_str, tok_box);
+  if (frame_mode) {
+    tm_kc = tm_k;   // not read
+    tm_vc = tm_v;
+  } else {
+    const uint64_t c_dims[3] = {static_cast<uint64_t>(pl.d), static_cast<uint64_t>(pl.M), static_cast<uint64_t>(pl.H)};
+    const uint64_t c_str[2] = {static_cast<uint64_t>(pl.d) * 2, static_cast<uint64_t>(pl.M) * pl.d * 2};
+    const uint32_t c_box[3] = {kHeadDim, kTileKV, 1};
+    good = good && make_tmap_bf16(&tm_kc, Kc, 3, c_dims, c_str, c_box);
+    good = good && make_tmap_bf16(&tm_vc, Vc, 3, c_dims, c_str, c_box);
+  }
   if (!good) { *tmap_failed = true; return cudaSuccess; }
 
   cudaError_t e = cudaMemsetAsync(ws, 0, kAttnStatusBytes, st);
@@ -769,9 +805,24 @@ cudaError_t launch_global_attn(const Plan& pl, int /*sm_count*/, const void* Q, 
   e = cudaFuncSetAttribute(global_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kAttnSmemBytes));
   if (e != cudaSuccess) return e;
   const int rows_per_cta = kQTiles * kTileQ;
-  const dim3 grid(static_cast<unsigned>((pl.n_tok + rows_per_cta - 1) / rows_per_cta), static_cast<unsigned>(pl.H));
+  const int64_t rows = frame_mode ? pl.L : pl.n_tok;
+  const dim3 grid(static_cast<unsigned>((rows + rows_per_cta - 1) / rows_per_cta), static_cast<unsigned>(pl.H),
+                  frame_mode ? static_cast<unsigned>(pl.n_frames) : 1u);
   global_attn_kernel<<<grid, kThreads, kAttnSmemBytes, st>>>(tm_q, tm_k, tm_v, tm_kc, tm_vc, a);
   return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_global_attn(const Plan& pl, int /*sm_count*/, const void* Q, const void* K, const void* V,
+                               const void* Kc, const void* Vc, const float* kmean, const float* vmean, void* O,
+                               float* lse, void* ws, cudaStream_t st, bool* tmap_failed) {
+  return launch_attn(pl, false, Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws, st, tmap_failed);
+}
+
+cudaError_t launch_frame_attn(const Plan& pl, const void* Q, const void* K, const void* V, void* O, float* lse, void* ws,
+                              cudaStream_t st, bool* tmap_failed) {
+  return launch_attn(pl, true, Q, K, V, nullptr, nullptr, nullptr, nullptr, O, lse, ws, st, tmap_failed);
 }
 
 }  // namespace avggt

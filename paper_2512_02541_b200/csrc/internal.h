@@ -23,4 +23,8 @@ cudaError_t launch_global_attn(const Plan& pl, int sm_count, const void* Q, cons
                                const void* Kc, const void* Vc, const float* kmean, const float* vmean, void* O,
                                float* lse, void* ws, cudaStream_t st, bool* tmap_failed);
 
+// Frame attention (Sec. 4.2): the same kernel, one independent dense problem per frame.
+cudaError_t launch_frame_attn(const Plan& pl, const void* Q, const void* K, const void* V, void* O, float* lse, void* ws,
+                              cudaStream_t st, bool* tmap_failed);
+
 }  // namespace avggt

@@ -46,6 +46,15 @@ class SubsampledGlobalAttention:
                             self.attn_ws, self.attn_ws.numel(), self._stream())
         return out
 
+    def frame_attend(self, Q, K, V, out=None):
+        """Frame attention (a converted early global block): each frame attends to itself only."""
+        self._check_inputs(Q, K, V)
+        if out is None:
+            out = torch.empty_like(Q)
+        with torch.cuda.device(self.device):
+            B.avggt_frame_attn(self.params, Q, K, V, out, self.lse, self.attn_ws, self.attn_ws.numel(), self._stream())
+        return out
+
     def forward(self, Q, K, V, out=None):
         self._check_inputs(Q, K, V)
         with torch.cuda.device(self.device):
