@@ -162,8 +162,6 @@ template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setma
 // Optional per-phase cycle counters of the softmax loop (a tuning aid; compiled out by default).
 #ifdef AVGGT_PHASE_TIMERS
 __device__ unsigned long long g_phase_cycles[4][4][8];   // [softmax warpgroup][warp][phase], CTA (0, 0)
-__device__ long long g_trace[64];
-#define AVGGT_TRACE(cond, slot) do { if ((cond) && blockIdx.x == 3 && blockIdx.y == 0) g_trace[slot] = clock64(); } while (0)
 struct PhaseTimers {
   unsigned long long acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
   long long last = 0;
@@ -171,7 +169,6 @@ struct PhaseTimers {
   __device__ __forceinline__ void lap(int i) { const long long now = clock64(); acc[i] += now - last; last = now; }
 };
 #else
-#define AVGGT_TRACE(cond, slot) do { } while (0)
 struct PhaseTimers {
   __device__ __forceinline__ void start() {}
   __device__ __forceinline__ void lap(int) {}
@@ -270,7 +267,6 @@ __device__ __forceinline__ void issue_qk(const AttnArgs& a, Barriers* bars, uint
   if (elect_one()) {
     constexpr uint32_t idesc = umma_idesc_bf16(kTileQ, kTileKV, false);
     const uint64_t desc_k = umma_desc_sw128(k_base + stage * kTileBytes);
-    AVGGT_TRACE(j == 101, 16 + t);
 #pragma unroll
     for (int k = 0; k < kHeadDim / 16; ++k)
       umma_ss(tmem + t * kTmemTileStride, desc_q + (k * 32 >> 4), desc_k + (k * 32 >> 4), idesc, k > 0);
@@ -285,7 +281,6 @@ __device__ __forceinline__ void issue_pv(const AttnArgs& a, Barriers* bars, uint
   if (elect_one()) {
     constexpr uint32_t idesc = umma_idesc_bf16(kTileQ, kHeadDim, true);
     const uint64_t desc_v = umma_desc_sw128(v_base + stage * kTileBytes);
-    AVGGT_TRACE(j == 100, 18 + t);
 #pragma unroll
     for (int k = 0; k < kTileKV / 16; ++k)
       umma_ts(tmem + t * kTmemTileStride + kColO, tmem + t * kTmemTileStride + kColP + k * 8, desc_v + (k * 2048 >> 4),
@@ -312,17 +307,13 @@ __device__ __forceinline__ void mma_role(const AttnArgs& a, Barriers* bars, cons
   uint32_t k_parity = 0, v_parity = 0;   // parity of their "full" phase
   for (int j = 0; j < n_kv; ++j) {
     if (j + 1 < n_kv) {
-      AVGGT_TRACE(j == 100 && elect_one(), 40 + t);
       if (!wait_bar_warp(&bars->s_free[t], j & 1, bars, a, 22 + t, j)) return;
-      AVGGT_TRACE(j == 100 && elect_one(), 42 + t);
       if (!wait_bar_warp(&bars->k_full[k_stage], k_parity, bars, a, 24 + t, j)) return;
       tc_fence_after();
       issue_qk<t>(a, bars, tmem, desc_q, k_base, k_stage, j + 1);
       if (++k_stage == kStages) { k_stage = 0; k_parity ^= 1; }
     }
-    AVGGT_TRACE(j == 100 && elect_one(), 46 + t);
     if (!wait_bar_warp(&bars->p_full[t], j & 1, bars, a, 26 + t, j)) return;
-    AVGGT_TRACE(j == 100 && elect_one(), 48 + t);
     if (!wait_bar_warp(&bars->v_full[v_stage], v_parity, bars, a, 28 + t, j)) return;
     tc_fence_after();
     issue_pv<t>(a, bars, tmem, v_base, v_stage, j);
@@ -748,12 +739,9 @@ constexpr size_t kAttnSmemBytes = static_cast<size_t>(kTileBytes) * (kQTiles + 2
 size_t global_attn_ws_bytes(const Plan&, int) { return kAttnStatusBytes; }
 
 #ifdef AVGGT_PHASE_TIMERS
-// Tuning aids: copy the 4 x 4 x 8 phase counters / the 64 event stamps of the last launch to the host.
+// Tuning aid: copies the 4 x 4 x 8 phase counters of the last launch to the host.
 extern "C" int avggt_debug_phase_cycles(unsigned long long* out64) {
   return cudaMemcpyFromSymbol(out64, g_phase_cycles, sizeof(g_phase_cycles)) == cudaSuccess ? 0 : -1;
-}
-extern "C" int avggt_debug_trace(long long* out64) {
-  return cudaMemcpyFromSymbol(out64, g_trace, sizeof(g_trace)) == cudaSuccess ? 0 : -1;
 }
 #endif
 
