@@ -318,3 +318,57 @@ def frame_attn(cfg, Q, K, V, rows=None, return_lse=False):
         lse[out_i] = (mx + np.log(z))[:, 0]
     return (O, lse) if return_lse else O
 
+
+def global_attn_indexed(cfg, idx, Q, K, V, rows=None, return_lse=False):
+    """The same layer with a caller-chosen retained set (the alternative selectors of the
+    supplement, "Comparison with other subsampling strategies": random, high/low-norm or feature
+    based picks instead of the fixed grid).  ``idx`` lists the retained token indices (any order,
+    no repeats; the caller includes the special tokens it wants kept).  D is every token not in
+    ``idx``; everything else follows Sec. 4.3 exactly as in ``global_attn``: logits over the
+    retained set, the query's own column if it is in D (diag), one mean pair over D entering with
+    weight 1 or with the count of columns it stands for (mean_fill 1 / 2), one shared softmax.
+    The retained keys are taken in ascending token order.
+    """
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    H, d = cfg.n_heads, cfg.head_dim
+    assert Q.shape == (cfg.n_tokens, H, d) and K.shape == Q.shape and V.shape == Q.shape
+    idx = np.sort(np.asarray(idx, dtype=np.int64))
+    assert len(idx) > 0 and len(np.unique(idx)) == len(idx) and idx[0] >= 0 and idx[-1] < cfg.n_tokens
+    scale = cfg.scale
+    dropped = np.ones(cfg.n_tokens, dtype=bool)
+    dropped[idx] = False
+    n_dropped = int(dropped.sum())
+    Kc, Vc = K[idx], V[idx]                               # [M, H, d]
+    kmean = K[dropped].mean(axis=0) if n_dropped else None
+    vmean = V[dropped].mean(axis=0) if n_dropped else None
+    if rows is None:
+        rows = np.arange(cfg.n_tokens)
+    rows = np.asarray(rows, dtype=np.int64)
+    O = np.empty((len(rows), H, d), dtype=np.float64)
+    lse = np.empty((len(rows), H), dtype=np.float64)
+    for out_i, i in enumerate(rows):
+        q = Q[i]
+        parts = [scale * np.einsum("hd,mhd->hm", q, Kc)]
+        vals = [Vc.transpose(1, 0, 2)]                    # [H, M, d]
+        has_diag = bool(cfg.diag) and bool(dropped[i])
+        if has_diag:
+            parts.append((scale * np.einsum("hd,hd->h", q, K[i]))[:, None])
+            vals.append(V[i][:, None, :])
+        count = n_dropped - (1 if has_diag else 0)
+        if cfg.mean_fill != 0 and count > 0:
+            lm = scale * np.einsum("hd,hd->h", q, kmean)
+            if cfg.mean_fill == 2:
+                lm = lm + math.log(count)
+            parts.append(lm[:, None])
+            vals.append(vmean[:, None, :])
+        logits = np.concatenate(parts, axis=1)
+        values = np.concatenate(vals, axis=1)             # [H, cols, d]
+        mx = logits.max(axis=1, keepdims=True)
+        p = np.exp(logits - mx)
+        z = p.sum(axis=1, keepdims=True)
+        O[out_i] = np.einsum("hc,hcd->hd", p / z, values)
+        lse[out_i] = (mx + np.log(z))[:, 0]
+    return (O, lse) if return_lse else O
+

@@ -54,10 +54,11 @@ def _dropped_by_slicing(cfg):
     return out.reshape(-1)
 
 
-def _brute_force(cfg, Q, K, V):
+def _brute_force(cfg, Q, K, V, D=None):
     n_tok, H, d = Q.shape
     scale = 1.0 / math.sqrt(d) if cfg.softmax_scale <= 0 else cfg.softmax_scale
-    D = _dropped_by_slicing(cfg)
+    if D is None:
+        D = _dropped_by_slicing(cfg)
     O = np.zeros((n_tok, H, d))
     for h in range(H):
         if D.any():
@@ -374,3 +375,38 @@ def test_frame_attn_rows_and_switches():
     rows = np.array([0, 12, 13, 25, 38])
     np.testing.assert_array_equal(orc.frame_attn(a, Q, K, V, rows=rows), full[rows])
     np.testing.assert_array_equal(orc.frame_attn(b, Q, K, V), full)
+
+
+# --------------------------------------------------------------------------
+# caller-chosen retained set (the supplement's alternative selectors)
+# --------------------------------------------------------------------------
+
+@pytest.mark.parametrize("sigma", (2, 6))
+@pytest.mark.parametrize("diag,mean_fill", [(False, 0), (True, 0), (False, 2), (True, 2), (True, 1)])
+def test_indexed_with_the_grid_subset_is_the_grid_layer(sigma, diag, mean_fill):
+    cfg = _tiny(sigma, diag, mean_fill)
+    Q, K, V = _rand_qkv(cfg, seed=31 + sigma)
+    got, lse = orc.global_attn_indexed(cfg, orc.build_index(cfg), Q, K, V, return_lse=True)
+    want, want_lse = orc.global_attn(cfg, Q, K, V, return_lse=True)
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(lse, want_lse, rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("diag,mean_fill", list(itertools.product((False, True), (0, 1, 2))))
+def test_indexed_random_subset_matches_filled_matrix_brute_force(diag, mean_fill):
+    cfg = _tiny(4, diag, mean_fill)
+    Q, K, V = _rand_qkv(cfg, seed=41 + 2 * int(diag) + mean_fill)
+    rng = np.random.default_rng(7)
+    idx = rng.permutation(cfg.n_tokens)[:17]              # unsorted on purpose; drops special tokens too
+    D = np.ones(cfg.n_tokens, dtype=bool)
+    D[idx] = False
+    np.testing.assert_allclose(orc.global_attn_indexed(cfg, idx, Q, K, V), _brute_force(cfg, Q, K, V, D=D), rtol=0, atol=1e-12)
+
+
+def test_indexed_keeping_everything_is_dense_sdpa():
+    cfg = orc.SGAConfig(2, 3, 4, 1, 2, 8, sigma=9, diag=True, mean_fill=2)
+    Q, K, V = _rand_qkv(cfg, seed=51)
+    tq, tk, tv = (torch.from_numpy(a).permute(1, 0, 2)[None] for a in (Q, K, V))
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv)[0].permute(1, 0, 2).numpy()
+    np.testing.assert_allclose(orc.global_attn_indexed(cfg, np.arange(cfg.n_tokens), Q, K, V), ref, rtol=0, atol=1e-12)
+
