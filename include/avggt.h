@@ -171,6 +171,33 @@ int avggt_global_attn(const avggt_params* p, const void* Q, const void* K, const
                       void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * The same layer with a retained set chosen by the caller instead of the window rule (the
+ * alternative selectors of the supplement, "Comparison with other subsampling strategies":
+ * random, norm-ranked or feature-based picks).  `idx` lists the n_kept retained tokens; every
+ * other token is in D, whatever its kind (list the special tokens to keep them).  Diagonal
+ * preservation, the mean pair over D and the shared softmax are as in Sec. 4.3.  Of `p`, sigma
+ * and flags play no part but must be valid.
+ *
+ * avggt_build_kv_indexed
+ *   idx            device, int32 [n_kept], strictly ascending token indices in [0, N*L).  The list
+ *                  is not checked on the host: entries out of range are skipped, a repeated entry
+ *                  leaves one compact row unwritten; neither reads or writes out of bounds.
+ *   K, V, Kc, Vc, kmean, vmean, ws   as for avggt_build_kv, with M = n_kept
+ *   slot_of_token  device, int32 [N*L]              written: compact position of a retained
+ *                  token, -1 for a dropped one.  Pass it on to avggt_global_attn_indexed.
+ * avggt_global_attn_indexed
+ *   as avggt_global_attn with M = n_kept and the map from avggt_build_kv_indexed.
+ */
+int avggt_build_kv_indexed(const avggt_params* p, const int32_t* idx, int64_t n_kept,
+                           const void* K, const void* V, void* Kc, void* Vc,
+                           int32_t* slot_of_token, float* kmean, float* vmean,
+                           void* ws, size_t ws_bytes, void* cuda_stream);
+int avggt_global_attn_indexed(const avggt_params* p, int64_t n_kept, const int32_t* slot_of_token,
+                              const void* Q, const void* K, const void* V,
+                              const void* Kc, const void* Vc, const float* kmean, const float* vmean,
+                              void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * Frame attention of a converted early global block (Sec. 4.2, "Global-to-Frame Attention
  * Conversion"): the (B, N L, C) rearrangement is skipped, so every token attends to the L tokens
  * of its own frame only, special tokens included, with plain softmax attention:

@@ -25,7 +25,7 @@ AVGGT_MEAN_OFF, AVGGT_MEAN_UNIT, AVGGT_MEAN_FILL = 0, 1, 2
 # every symbol include/avggt.h declares
 EXPORTS = (
     "avggt_kv_count", "avggt_workspace_bytes", "avggt_build_kv", "avggt_build_kv_noalloc", "avggt_global_attn",
-    "avggt_frame_attn",
+    "avggt_frame_attn", "avggt_build_kv_indexed", "avggt_global_attn_indexed",
     "avggt_check_status", "avggt_strerror", "avggt_last_cuda_error", "avggt_version",
 )
 
@@ -85,6 +85,10 @@ def lib():
         L.avggt_global_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.avggt_frame_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.avggt_frame_attn.restype = ctypes.c_int
+        L.avggt_build_kv_indexed.argtypes = [pp, vp, ctypes.c_int64, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.avggt_build_kv_indexed.restype = ctypes.c_int
+        L.avggt_global_attn_indexed.argtypes = [pp, ctypes.c_int64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.avggt_global_attn_indexed.restype = ctypes.c_int
         L.avggt_check_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
         L.avggt_strerror.argtypes = [ctypes.c_int]
         for f in (L.avggt_kv_count, L.avggt_workspace_bytes, L.avggt_build_kv, L.avggt_global_attn, L.avggt_check_status):
@@ -150,6 +154,21 @@ def avggt_global_attn(params, Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws, ws_byte
     """Enqueue the subsampled global attention."""
     _check(lib().avggt_global_attn(ctypes.byref(params), _ptr(Q), _ptr(K), _ptr(V), _ptr(Kc), _ptr(Vc), _ptr(kmean),
                                    _ptr(vmean), _ptr(O), _ptr(lse), _ptr(ws), ws_bytes, stream), "avggt_global_attn")
+
+
+def avggt_build_kv_indexed(params, idx, n_kept, K, V, Kc, Vc, slot_of_token, kmean, vmean, ws, ws_bytes, stream=None):
+    """Enqueue the compaction + mean reduction for a caller-chosen retained set (ascending int32 token indices)."""
+    _check(lib().avggt_build_kv_indexed(ctypes.byref(params), _ptr(idx), n_kept, _ptr(K), _ptr(V), _ptr(Kc), _ptr(Vc),
+                                        _ptr(slot_of_token), _ptr(kmean), _ptr(vmean), _ptr(ws), ws_bytes, stream),
+           "avggt_build_kv_indexed")
+
+
+def avggt_global_attn_indexed(params, n_kept, slot_of_token, Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws, ws_bytes,
+                              stream=None):
+    """Enqueue the attention over a caller-chosen retained set."""
+    _check(lib().avggt_global_attn_indexed(ctypes.byref(params), n_kept, _ptr(slot_of_token), _ptr(Q), _ptr(K), _ptr(V),
+                                           _ptr(Kc), _ptr(Vc), _ptr(kmean), _ptr(vmean), _ptr(O), _ptr(lse), _ptr(ws),
+                                           ws_bytes, stream), "avggt_global_attn_indexed")
 
 
 def avggt_frame_attn(params, Q, K, V, O, lse, ws, ws_bytes, stream=None):

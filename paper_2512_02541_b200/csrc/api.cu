@@ -169,6 +169,66 @@ int avggt_global_attn(const avggt_params* p, const void* Q, const void* K, const
   return record_cuda(e);
 }
 
+// Plan of a problem whose retained set is a caller-supplied list of n_kept tokens.
+static int make_indexed_plan(const avggt_params* p, int64_t n_kept, Plan* pl) {
+  int rc = make_plan(p, pl);
+  if (rc != AVGGT_OK) return rc;
+  if (n_kept < 1 || n_kept > pl->n_tok) return AVGGT_ERR_INVALID_ARG;
+  pl->M = n_kept;
+  pl->n_dropped = pl->n_tok - n_kept;
+  pl->keep_first = 0;
+  return AVGGT_OK;
+}
+
+int avggt_build_kv_indexed(const avggt_params* p, const int32_t* idx, int64_t n_kept, const void* K, const void* V,
+                           void* Kc, void* Vc, int32_t* slot_of_token, float* kmean, float* vmean, void* ws,
+                           size_t ws_bytes, void* cuda_stream) {
+  Plan pl;
+  int rc = make_indexed_plan(p, n_kept, &pl);
+  if (rc != AVGGT_OK) return rc;
+  if (!idx || !slot_of_token || !K || !V || !Kc || !Vc || !ws) return AVGGT_ERR_INVALID_ARG;
+  if (pl.mean_fill != 0 && (!kmean || !vmean)) return AVGGT_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(V) || !aligned16(Kc) || !aligned16(Vc) || !aligned16(ws) ||
+      (reinterpret_cast<uintptr_t>(idx) & 3u) || (reinterpret_cast<uintptr_t>(slot_of_token) & 3u) ||
+      !aligned16(kmean) || !aligned16(vmean))
+    return AVGGT_ERR_ALIGNMENT;
+  DeviceInfo di;
+  rc = device_info(&di);
+  if (rc != AVGGT_OK) return rc;
+  if (ws_bytes < build_kv_ws_bytes(pl, di.sm_count)) return AVGGT_ERR_WORKSPACE_TOO_SMALL;
+  return record_cuda(launch_build_kv(pl, di.sm_count, K, V, Kc, Vc, nullptr, kmean, vmean, ws,
+                                     static_cast<cudaStream_t>(cuda_stream), idx, slot_of_token));
+}
+
+int avggt_global_attn_indexed(const avggt_params* p, int64_t n_kept, const int32_t* slot_of_token, const void* Q,
+                              const void* K, const void* V, const void* Kc, const void* Vc, const float* kmean,
+                              const float* vmean, void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Plan pl;
+  int rc = make_indexed_plan(p, n_kept, &pl);
+  if (rc != AVGGT_OK) return rc;
+  const bool need_diag = pl.diag != 0 && pl.n_dropped > 0;
+  const bool need_mean = pl.mean_fill != 0 && pl.n_dropped > 0;
+  if (!Q || !Kc || !Vc || !O || !ws || !slot_of_token) return AVGGT_ERR_INVALID_ARG;
+  if (need_diag && (!K || !V)) return AVGGT_ERR_INVALID_ARG;
+  if (need_mean && (!kmean || !vmean)) return AVGGT_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(Kc) || !aligned16(Vc) || !aligned16(O) ||
+      !aligned16(ws) || !aligned16(kmean) || !aligned16(vmean) || (reinterpret_cast<uintptr_t>(lse) & 3u) ||
+      (reinterpret_cast<uintptr_t>(slot_of_token) & 3u))
+    return AVGGT_ERR_ALIGNMENT;
+  DeviceInfo di;
+  rc = device_info(&di);
+  if (rc != AVGGT_OK) return rc;
+  if (ws_bytes < global_attn_ws_bytes(pl, di.sm_count)) return AVGGT_ERR_WORKSPACE_TOO_SMALL;
+  bool tmap_failed = false;
+  cudaError_t e = launch_global_attn(pl, di.sm_count, Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws,
+                                     static_cast<cudaStream_t>(cuda_stream), &tmap_failed, slot_of_token);
+  if (tmap_failed) {
+    std::strncpy(g_cuda_error, "cuTensorMapEncodeTiled failed", sizeof(g_cuda_error) - 1);
+    return AVGGT_ERR_CUDA;
+  }
+  return record_cuda(e);
+}
+
 int avggt_frame_attn(const avggt_params* p, const void* Q, const void* K, const void* V, void* O, float* lse, void* ws,
                      size_t ws_bytes, void* cuda_stream) {
   Plan pl;

@@ -42,7 +42,8 @@ __device__ __forceinline__ void add_bf16x8(float (&acc)[8], const uint4& v) {
 template <int PASSES>
 __global__ void __launch_bounds__(kBuildThreads)
 build_kv_kernel(const Plan pl, const uint4* __restrict__ K, const uint4* __restrict__ V, uint4* __restrict__ Kc,
-                uint4* __restrict__ Vc, int32_t* __restrict__ idx, float* __restrict__ partials, const int do_mean) {
+                uint4* __restrict__ Vc, int32_t* __restrict__ idx, float* __restrict__ partials, const int do_mean,
+                const int32_t* __restrict__ slot_of_token) {
   extern __shared__ float red[];   // [kBuildWarps][PASSES * 256]
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
@@ -59,7 +60,9 @@ build_kv_kernel(const Plan pl, const uint4* __restrict__ K, const uint4* __restr
   for (uint32_t row = blockIdx.x * kBuildWarps + warp; row < n_tok; row += warps_total) {
     const int32_t f = static_cast<int32_t>(row / static_cast<uint32_t>(pl.L));
     const int32_t u = static_cast<int32_t>(row - static_cast<uint32_t>(f) * static_cast<uint32_t>(pl.L));
-    const int32_t cs = compact_slot(pl, f, u);
+    // compact position within the frame's block by the window rule, or, for a caller-chosen retained set,
+    // the global compact position from the caller's map
+    const int32_t cs = slot_of_token != nullptr ? slot_of_token[row] : compact_slot(pl, f, u);
     if (cs < 0 && !do_mean) continue;
     const uint4* krow = K + static_cast<size_t>(row) * chunks_per_row;
     const uint4* vrow = V + static_cast<size_t>(row) * chunks_per_row;
@@ -71,7 +74,7 @@ build_kv_kernel(const Plan pl, const uint4* __restrict__ K, const uint4* __restr
       else { kv[p] = make_uint4(0, 0, 0, 0); vv[p] = make_uint4(0, 0, 0, 0); }
     }
     if (cs >= 0) {
-      const int64_t m = compact_frame_base(pl, f) + cs;
+      const int64_t m = slot_of_token != nullptr ? cs : compact_frame_base(pl, f) + cs;
       if (lane == 0 && idx != nullptr) idx[m] = static_cast<int32_t>(row);
 #pragma unroll
       for (int p = 0; p < PASSES; ++p) {
@@ -134,16 +137,32 @@ mean_finalize_kernel(const float* __restrict__ partials, int n_blocks, int cols2
   }
 }
 
+// slot_of_token[t] = -1 for every token, then m for the m-th retained token.  Entries of idx outside
+// [0, n_tok) are skipped.
+__global__ void fill_slots_kernel(int32_t* __restrict__ slot_of_token, int64_t n_tok) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < n_tok) slot_of_token[i] = -1;
+}
+__global__ void scatter_slots_kernel(const int32_t* __restrict__ idx, int64_t M, int32_t* __restrict__ slot_of_token,
+                                     int64_t n_tok) {
+  const int64_t m = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (m < M) {
+    const int32_t t = idx[m];
+    if (t >= 0 && t < n_tok) slot_of_token[t] = static_cast<int32_t>(m);
+  }
+}
+
 template <int PASSES>
 cudaError_t launch_build(const Plan& pl, int grid, const void* K, const void* V, void* Kc, void* Vc, int32_t* idx,
-                         float* partials, int do_mean, cudaStream_t st) {
+                         float* partials, int do_mean, const int32_t* slot_of_token, cudaStream_t st) {
   const size_t smem = do_mean ? static_cast<size_t>(kBuildWarps) * PASSES * 256 * sizeof(float) : 0;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(build_kv_kernel<PASSES>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
   }
   build_kv_kernel<PASSES><<<grid, kBuildThreads, smem, st>>>(pl, static_cast<const uint4*>(K), static_cast<const uint4*>(V),
-                                                           static_cast<uint4*>(Kc), static_cast<uint4*>(Vc), idx, partials, do_mean);
+                                                           static_cast<uint4*>(Kc), static_cast<uint4*>(Vc), idx, partials, do_mean,
+                                                           slot_of_token);
   return cudaGetLastError();
 }
 
@@ -162,21 +181,30 @@ size_t build_kv_ws_bytes(const Plan& pl, int sm_count) {
 }
 
 cudaError_t launch_build_kv(const Plan& pl, int sm_count, const void* K, const void* V, void* Kc, void* Vc,
-                            int32_t* idx, float* kmean, float* vmean, void* ws, cudaStream_t st) {
+                            int32_t* idx, float* kmean, float* vmean, void* ws, cudaStream_t st,
+                            const int32_t* caller_idx, int32_t* slot_of_token) {
+  if (caller_idx != nullptr) {
+    // caller-chosen retained set: build the token -> compact position map first
+    fill_slots_kernel<<<static_cast<unsigned>((pl.n_tok + 255) / 256), 256, 0, st>>>(slot_of_token, pl.n_tok);
+    scatter_slots_kernel<<<static_cast<unsigned>((pl.M + 255) / 256), 256, 0, st>>>(caller_idx, pl.M, slot_of_token, pl.n_tok);
+    cudaError_t e0 = cudaGetLastError();
+    if (e0 != cudaSuccess) return e0;
+    idx = nullptr;
+  }
   const int grid = build_kv_grid(pl, sm_count);
   const int do_mean = (pl.mean_fill != 0 && pl.n_dropped > 0) ? 1 : 0;
   float* partials = static_cast<float*>(ws);
   const int passes = (pl.H * 8 + 31) / 32;
   cudaError_t e;
   switch (passes) {
-    case 1: e = launch_build<1>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, st); break;
-    case 2: e = launch_build<2>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, st); break;
-    case 3: e = launch_build<3>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, st); break;
-    case 4: e = launch_build<4>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, st); break;
-    case 5: e = launch_build<5>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, st); break;
-    case 6: e = launch_build<6>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, st); break;
-    case 7: e = launch_build<7>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, st); break;
-    case 8: e = launch_build<8>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, st); break;
+    case 1: e = launch_build<1>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, slot_of_token, st); break;
+    case 2: e = launch_build<2>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, slot_of_token, st); break;
+    case 3: e = launch_build<3>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, slot_of_token, st); break;
+    case 4: e = launch_build<4>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, slot_of_token, st); break;
+    case 5: e = launch_build<5>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, slot_of_token, st); break;
+    case 6: e = launch_build<6>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, slot_of_token, st); break;
+    case 7: e = launch_build<7>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, slot_of_token, st); break;
+    case 8: e = launch_build<8>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, slot_of_token, st); break;
     default: return cudaErrorInvalidValue;
   }
   if (e != cudaSuccess) return e;

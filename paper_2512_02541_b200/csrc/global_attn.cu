@@ -75,6 +75,7 @@ struct AttnArgs {
   const float* vmean;
   __nv_bfloat16* O;     // [n_tok, H, d]
   float* lse;           // [n_tok, H] or null
+  const int32_t* slot_of_token;   // caller-chosen retained set: compact position of every token, -1 = dropped; else null
   uint32_t* status;     // 4 words
   int32_t frame_mode;   // 0: subsampled global attention over the compact keys.  1: frame attention (Sec. 4.2):
                         //    blockIdx.z is the frame, keys and values are the frame's own rows of K and V
@@ -559,7 +560,7 @@ __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, 
   bool is_dropped = false;
   if (row_valid && pl.n_dropped > 0) {
     const int32_t f = row / pl.L;
-    is_dropped = compact_slot(pl, f, row - f * pl.L) < 0;
+    is_dropped = (a.slot_of_token != nullptr ? a.slot_of_token[row] : compact_slot(pl, f, row - f * pl.L)) < 0;
   }
   // the row's sums: mine plus the partner's
   px->final[t][0][me.h][r] = l_run;
@@ -750,10 +751,11 @@ namespace {
 // Tensor maps and launch shared by the two entry points.  frame_mode: see AttnArgs.
 cudaError_t launch_attn(const Plan& pl, bool frame_mode, const void* Q, const void* K, const void* V, const void* Kc,
                         const void* Vc, const float* kmean, const float* vmean, void* O, float* lse, void* ws,
-                        cudaStream_t st, bool* tmap_failed) {
+                        cudaStream_t st, bool* tmap_failed, const int32_t* slot_of_token) {
   *tmap_failed = false;
   AttnArgs a;
   a.pl = pl;
+  a.slot_of_token = slot_of_token;
   a.kmean = kmean;
   a.vmean = vmean;
   a.O = static_cast<__nv_bfloat16*>(O);
@@ -804,13 +806,13 @@ cudaError_t launch_attn(const Plan& pl, bool frame_mode, const void* Q, const vo
 
 cudaError_t launch_global_attn(const Plan& pl, int /*sm_count*/, const void* Q, const void* K, const void* V,
                                const void* Kc, const void* Vc, const float* kmean, const float* vmean, void* O,
-                               float* lse, void* ws, cudaStream_t st, bool* tmap_failed) {
-  return launch_attn(pl, false, Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws, st, tmap_failed);
+                               float* lse, void* ws, cudaStream_t st, bool* tmap_failed, const int32_t* slot_of_token) {
+  return launch_attn(pl, false, Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws, st, tmap_failed, slot_of_token);
 }
 
 cudaError_t launch_frame_attn(const Plan& pl, const void* Q, const void* K, const void* V, void* O, float* lse, void* ws,
                               cudaStream_t st, bool* tmap_failed) {
-  return launch_attn(pl, true, Q, K, V, nullptr, nullptr, nullptr, nullptr, O, lse, ws, st, tmap_failed);
+  return launch_attn(pl, true, Q, K, V, nullptr, nullptr, nullptr, nullptr, O, lse, ws, st, tmap_failed, nullptr);
 }
 
 }  // namespace avggt
