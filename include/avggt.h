@@ -198,6 +198,25 @@ int avggt_global_attn_indexed(const avggt_params* p, int64_t n_kept, const int32
                               void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Subsampled global attention for a shard of the frames (one rank of a frame-sharded run): the
+ * queries are the tokens of the n_frames frames that `p` describes (this rank's), the compact keys
+ * and the mean pair are those of the WHOLE sequence (Sec. 4.3 defines S and the mean over all
+ * frames).  The caller gathers Kc/Vc of all ranks into one [H, n_kept_total, d] array in this
+ * GPU's memory and combines the ranks' means before the call; the library does no communication.
+ *
+ *   n_kept_total     compact keys of the whole sequence (>= this shard's own)
+ *   n_dropped_total  dropped tokens of the whole sequence (the count behind the mean pair)
+ *   Q, K, V, O, lse  this shard's rows only, [n_frames*L, H, d] / [n_frames*L, H]
+ *   Kc, Vc           device, bf16 [H, n_kept_total, d]
+ *   other arguments as for avggt_global_attn.  AVGGT_FLAG_KEEP_FIRST_FRAME refers to the first
+ *   frame of the shard: set it only on the rank that owns frame 0 of the sequence.
+ */
+int avggt_global_attn_shard(const avggt_params* p, int64_t n_kept_total, int64_t n_dropped_total,
+                            const void* Q, const void* K, const void* V,
+                            const void* Kc, const void* Vc, const float* kmean, const float* vmean,
+                            void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * Frame attention of a converted early global block (Sec. 4.2, "Global-to-Frame Attention
  * Conversion"): the (B, N L, C) rearrangement is skipped, so every token attends to the L tokens
  * of its own frame only, special tokens included, with plain softmax attention:

@@ -25,7 +25,7 @@ AVGGT_MEAN_OFF, AVGGT_MEAN_UNIT, AVGGT_MEAN_FILL = 0, 1, 2
 # every symbol include/avggt.h declares
 EXPORTS = (
     "avggt_kv_count", "avggt_workspace_bytes", "avggt_build_kv", "avggt_build_kv_noalloc", "avggt_global_attn",
-    "avggt_frame_attn", "avggt_build_kv_indexed", "avggt_global_attn_indexed",
+    "avggt_frame_attn", "avggt_build_kv_indexed", "avggt_global_attn_indexed", "avggt_global_attn_shard",
     "avggt_check_status", "avggt_strerror", "avggt_last_cuda_error", "avggt_version",
 )
 
@@ -89,6 +89,8 @@ def lib():
         L.avggt_build_kv_indexed.restype = ctypes.c_int
         L.avggt_global_attn_indexed.argtypes = [pp, ctypes.c_int64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.avggt_global_attn_indexed.restype = ctypes.c_int
+        L.avggt_global_attn_shard.argtypes = [pp, ctypes.c_int64, ctypes.c_int64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.avggt_global_attn_shard.restype = ctypes.c_int
         L.avggt_check_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
         L.avggt_strerror.argtypes = [ctypes.c_int]
         for f in (L.avggt_kv_count, L.avggt_workspace_bytes, L.avggt_build_kv, L.avggt_global_attn, L.avggt_check_status):
@@ -169,6 +171,14 @@ def avggt_global_attn_indexed(params, n_kept, slot_of_token, Q, K, V, Kc, Vc, km
     _check(lib().avggt_global_attn_indexed(ctypes.byref(params), n_kept, _ptr(slot_of_token), _ptr(Q), _ptr(K), _ptr(V),
                                            _ptr(Kc), _ptr(Vc), _ptr(kmean), _ptr(vmean), _ptr(O), _ptr(lse), _ptr(ws),
                                            ws_bytes, stream), "avggt_global_attn_indexed")
+
+
+def avggt_global_attn_shard(params, n_kept_total, n_dropped_total, Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws, ws_bytes,
+                            stream=None):
+    """Enqueue the attention of one frame shard against the whole sequence's compact keys and mean pair."""
+    _check(lib().avggt_global_attn_shard(ctypes.byref(params), n_kept_total, n_dropped_total, _ptr(Q), _ptr(K), _ptr(V),
+                                         _ptr(Kc), _ptr(Vc), _ptr(kmean), _ptr(vmean), _ptr(O), _ptr(lse), _ptr(ws),
+                                         ws_bytes, stream), "avggt_global_attn_shard")
 
 
 def avggt_frame_attn(params, Q, K, V, O, lse, ws, ws_bytes, stream=None):

@@ -229,6 +229,38 @@ int avggt_global_attn_indexed(const avggt_params* p, int64_t n_kept, const int32
   return record_cuda(e);
 }
 
+int avggt_global_attn_shard(const avggt_params* p, int64_t n_kept_total, int64_t n_dropped_total, const void* Q,
+                            const void* K, const void* V, const void* Kc, const void* Vc, const float* kmean,
+                            const float* vmean, void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Plan pl;
+  int rc = make_plan(p, &pl);
+  if (rc != AVGGT_OK) return rc;
+  // the shard's own frames cannot hold more retained or dropped tokens than the whole sequence
+  if (n_kept_total < pl.M || n_dropped_total < pl.n_dropped) return AVGGT_ERR_INVALID_ARG;
+  pl.M = n_kept_total;
+  pl.n_dropped = n_dropped_total;
+  const bool need_diag = pl.diag != 0 && pl.n_dropped > 0;
+  const bool need_mean = pl.mean_fill != 0 && pl.n_dropped > 0;
+  if (!Q || !Kc || !Vc || !O || !ws) return AVGGT_ERR_INVALID_ARG;
+  if (need_diag && (!K || !V)) return AVGGT_ERR_INVALID_ARG;
+  if (need_mean && (!kmean || !vmean)) return AVGGT_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(Kc) || !aligned16(Vc) || !aligned16(O) ||
+      !aligned16(ws) || !aligned16(kmean) || !aligned16(vmean) || (reinterpret_cast<uintptr_t>(lse) & 3u))
+    return AVGGT_ERR_ALIGNMENT;
+  DeviceInfo di;
+  rc = device_info(&di);
+  if (rc != AVGGT_OK) return rc;
+  if (ws_bytes < global_attn_ws_bytes(pl, di.sm_count)) return AVGGT_ERR_WORKSPACE_TOO_SMALL;
+  bool tmap_failed = false;
+  cudaError_t e = launch_global_attn(pl, di.sm_count, Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws,
+                                     static_cast<cudaStream_t>(cuda_stream), &tmap_failed);
+  if (tmap_failed) {
+    std::strncpy(g_cuda_error, "cuTensorMapEncodeTiled failed", sizeof(g_cuda_error) - 1);
+    return AVGGT_ERR_CUDA;
+  }
+  return record_cuda(e);
+}
+
 int avggt_frame_attn(const avggt_params* p, const void* Q, const void* K, const void* V, void* O, float* lse, void* ws,
                      size_t ws_bytes, void* cuda_stream) {
   Plan pl;

@@ -69,3 +69,46 @@ def test_reference_arm_prints_on_rank_zero_only():
     line = json.loads(res.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle" and line["value"] > 0
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["n_gpus"] == 2
+
+
+# --------------------------------------------------------------------------
+# frame-sharded layer: the exchange step (all-gather of compact K/V, all-reduce of the mean sums)
+# --------------------------------------------------------------------------
+
+def test_shard_frames_covers_all_frames_evenly():
+    from paper_2512_02541_b200.sharded import shard_frames
+    for n, w in [(100, 8), (7, 3), (8, 8), (333, 4), (5, 1)]:
+        ranges = [shard_frames(n, w, r) for r in range(w)]
+        assert ranges[0][0] == 0 and ranges[-1][1] == n
+        assert all(a[1] == b[0] for a, b in zip(ranges, ranges[1:]))
+        sizes = [f1 - f0 for f0, f1 in ranges]
+        assert max(sizes) - min(sizes) <= 1 and sizes == sorted(sizes, reverse=True)
+
+
+def _exchange_main(rank, world, port, out_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2512_02541_b200.sharded import combine_means, gather_compact
+    H, d = 3, 8
+    kept = [5, 9]                                  # uneven shards: padding on rank 0
+    dropped = [40, 24]
+    gen = torch.Generator().manual_seed(100 + rank)
+    local = torch.randn((H, kept[rank], d), generator=gen).bfloat16()
+    mean = torch.randn((H, d), generator=gen)
+    full = gather_compact(local, kept)
+    m, total = combine_means(mean, dropped[rank])
+    torch.save({"local": local, "mean": mean, "full": full, "m": m, "total": total}, os.path.join(out_dir, f"x{rank}.pt"))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_exchange_step_two_gloo_ranks(tmp_path):
+    world = 2
+    mp.spawn(_exchange_main, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    got = [torch.load(tmp_path / f"x{r}.pt") for r in range(world)]
+    want_full = torch.cat([got[0]["local"], got[1]["local"]], dim=1)          # rank order = ascending token order
+    want_mean = (got[0]["mean"].double() * 40 + got[1]["mean"].double() * 24) / 64
+    for r in range(world):
+        assert torch.equal(got[r]["full"], want_full)
+        assert got[r]["total"] == 64
+        assert torch.allclose(got[r]["m"].double(), want_mean, rtol=0, atol=1e-6)
