@@ -246,6 +246,26 @@ def run_ours(args, wl):
     layer.check_status()
     frame_ms = fe[0].elapsed_time(fe[1]) / args.steps
 
+    # ---- outside the timed region: the dense layer (s = 1, both switches off) on the same tokens, the GPU
+    #      reference the metric is quoted against
+    dense_ms = None
+    if wl.sigma != 1 and not args.no_dense:
+        dparams = P.make_params(wl.n_frames, wl.grid_h, wl.grid_w, wl.n_special, wl.n_heads, wl.head_dim, 1,
+                                diag=0, mean_fill=0)
+        dense = P.SubsampledGlobalAttention(dparams, device=dev)
+        dense.forward(Q, K, V, out=O)
+        barrier()
+        de = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        n_dense = 2
+        de[0].record(stream)
+        for _ in range(n_dense):
+            dense.attend(Q, K, V, out=O)
+        de[1].record(stream)
+        barrier()
+        dense.check_status()
+        dense_ms = de[0].elapsed_time(de[1]) / n_dense
+        del dense
+
     # ---- end to end through the public API with host buffers
     e2e_steps = max(1, min(args.steps, 5))
     hQ, hK, hV = (t.cpu().pin_memory() for t in (Q, K, V))
@@ -294,6 +314,8 @@ def run_ours(args, wl):
             "tflops": world * flops / (ms_per_step * 1e-3) / 1e12,
             "attn_ms": attn_avg, "attn_ms_min": min(attn_ms), "build_kv_ms": build_avg, "build_kv_ms_min": min(build_ms),
             "attn_queries_per_sec": n_q / (attn_avg * 1e-3),
+            "dense_attn_ms": dense_ms,
+            "speedup_vs_dense": (dense_ms / attn_avg) if dense_ms else None,
             "frame_attn_ms": frame_ms,
             "frame_attn_tflops": 4.0 * n_q * wl.tokens_per_frame * H * d / (frame_ms * 1e-3) / 1e12,
             "roofline": {"bound": "tensor", "kernel": "global_attn_kernel", "achieved": achieved_tf, "peak": peak_tf,
@@ -331,6 +353,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--cpu-rows", type=int, default=4096, help="query rows in the CPU-oracle baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-dense", action="store_true", help="skip the dense (s = 1) comparison run")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     wl = inputs.WORKLOADS[args.workload]
