@@ -201,3 +201,24 @@ def test_argument_errors_do_not_launch():
                             layer.attn_ws, layer.attn_ws.numel())
     assert ei.value.code == -1
     torch.cuda.synchronize()
+
+
+def _random_workloads(n, seed=2024):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        out.append(inputs.Workload(
+            f"fuzz{i}", int(rng.integers(1, 7)), int(rng.integers(1, 24)), int(rng.integers(1, 24)),
+            int(rng.integers(0, 7)), int(rng.choice([1, 2, 3, 5, 8, 16, 32])), 64, int(rng.choice([1, 2, 4, 6, 9])),
+            int(rng.integers(0, 2)), int(rng.integers(0, 3)), str(rng.choice(["iid", "proj"])),
+            keep_first_frame=int(rng.integers(0, 2))))
+    return out
+
+
+@pytest.mark.parametrize("wl", _random_workloads(16), ids=lambda w: f"{w.name}-N{w.n_frames}-g{w.grid_h}x{w.grid_w}-s{w.n_special}-H{w.n_heads}-sig{w.sigma}-d{w.diag}-m{w.mean_fill}-k{w.keep_first_frame}")
+def test_seeded_random_shapes(wl):
+    """Sixteen seeded draws over frames, grid, special tokens, heads, factor, switches, value recipe and
+    the first-frame flag: compaction exact, attention and log-sum-exp within tolerance on every row."""
+    params, ocfg, layer, Q, K, V, O = _run_gpu(wl, seed=17, want_lse=True)
+    Kh, Vh = _check_build(ocfg, layer, K, V)
+    _check_attn(ocfg, Q, Kh, Vh, O, lse=layer.lse)
