@@ -36,7 +36,7 @@ from paper_2512_02541_b200 import inputs  # noqa: E402
 # profiles/; None where no capture covers the workload.  The attention kernel is captured on the 30-frame copy of
 # the layer (profiles/global_attn_kernel_vggt_n30_s4.md); its traffic is proportional to the frame count, so the
 # 100-frame figure is that capture x 100/30.  The compaction kernel is captured on the 100-frame workload itself.
-_ATTN_N30 = 0.299476e9 + 0.071481e9
+_ATTN_N30 = 0.299442e9 + 0.068250e9
 NCU_TRAFFIC = {
     "vggt_n30_s4": {"global_attn_kernel": _ATTN_N30},
     "vggt_n100_s4": {"global_attn_kernel": _ATTN_N30 * 100 / 30, "build_kv_kernel": 0.562812e9 + 0.104510e9},
