@@ -39,7 +39,7 @@ from paper_2512_02541_b200 import inputs  # noqa: E402
 _ATTN_N30 = 0.299442e9 + 0.068250e9
 NCU_TRAFFIC = {
     "vggt_n30_s4": {"global_attn_kernel": _ATTN_N30},
-    "vggt_n100_s4": {"global_attn_kernel": _ATTN_N30 * 100 / 30, "build_kv_kernel": 0.562812e9 + 0.104510e9},
+    "vggt_n100_s4": {"global_attn_kernel": _ATTN_N30 * 100 / 30, "build_kv_kernel": 0.562844e9 + 0.103259e9},
 }
 
 METRIC = "subsampled_global_attn_queries_per_sec"
