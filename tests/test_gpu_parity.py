@@ -222,3 +222,41 @@ def test_seeded_random_shapes(wl):
     params, ocfg, layer, Q, K, V, O = _run_gpu(wl, seed=17, want_lse=True)
     Kh, Vh = _check_build(ocfg, layer, K, V)
     _check_attn(ocfg, Q, Kh, Vh, O, lse=layer.lse)
+
+
+@pytest.mark.parametrize("scale", (0.05, 0.3))
+def test_caller_given_softmax_scale(scale):
+    """A softmax scale other than 1/sqrt(d), in both the global and the frame entry points."""
+    wl = inputs.Workload("scale", 3, 9, 9, 5, 4, 64, 4, 1, 2, "iid")
+    params = P.make_params(wl.n_frames, wl.grid_h, wl.grid_w, wl.n_special, wl.n_heads, wl.head_dim, wl.sigma,
+                           softmax_scale=scale)
+    ocfg = orc.SGAConfig(wl.n_frames, wl.grid_h, wl.grid_w, wl.n_special, wl.n_heads, wl.head_dim, wl.sigma,
+                         softmax_scale=scale)
+    Q, K, V = inputs.make_qkv(wl, seed=12, device="cuda")
+    layer = P.SubsampledGlobalAttention(params, want_lse=True)
+    O = layer.forward(Q, K, V)
+    layer.check_status()
+    Kh, Vh = _host(K), _host(V)
+    _check_attn(ocfg, Q, Kh, Vh, O, lse=layer.lse)
+    Of = layer.frame_attend(Q, K, V)
+    layer.check_status()
+    want = orc.frame_attn(ocfg, _host(Q), Kh, Vh)
+    err = np.abs(Of.float().cpu().numpy().astype(np.float64) - want)
+    assert err.max() <= MAX_ABS_TOL and err.mean() <= MEAN_ABS_TOL
+
+
+def test_extreme_values_stay_finite():
+    """Logits of a few hundred in magnitude with alternating sign between key tiles: the reference maximum
+    jumps late and far, the accumulator is rescaled by tiny factors, nothing overflows."""
+    wl = inputs.Workload("extreme", 4, 12, 12, 5, 2, 64, 2, 1, 2, "iid")
+    params, ocfg = _cfgs(wl)
+    Q, K, V = inputs.make_qkv(wl, seed=13, device="cuda")
+    K = (K.float() * 6.0).bfloat16()                      # scale * q.k of the order of +-150
+    L = wl.tokens_per_frame
+    K[2 * L:] = (K[2 * L:].float() * 2.0).bfloat16()      # later frames (later key tiles) reach further out
+    layer = P.SubsampledGlobalAttention(params, want_lse=True)
+    O = layer.forward(Q, K, V)
+    layer.check_status()
+    assert torch.isfinite(O.float()).all() and torch.isfinite(layer.lse).all()
+    Kh, Vh = _host(K), _host(V)
+    _check_attn(ocfg, Q, Kh, Vh, O, lse=None)
