@@ -21,8 +21,13 @@
  *     synchronising.  `cuda_stream` is a cudaStream_t passed as void*
  *     (NULL = the legacy default stream).
  *   - Return value: 0 on success, a negative AVGGT_ERR_* code otherwise.
- *     Arguments are validated on the host before anything is launched; on an
- *     error nothing has been enqueued.  No exception crosses this boundary.
+ *     Arguments are validated on the host before anything is launched; after an
+ *     argument error nothing has been enqueued.  (If the launch itself fails with
+ *     AVGGT_ERR_CUDA, the clearing of the status block may already be on the
+ *     stream; no kernel is.)  No exception crosses this boundary.
+ *   - Size limits: head_dim == 64; n_heads <= 32; batch == 1;
+ *     N * L <= 2^31 - 257 tokens; frame attention: N <= 65535 frames.  Anything
+ *     beyond them is rejected with AVGGT_ERR_UNSUPPORTED.
  *   - Only sm_100 devices are supported (AVGGT_ERR_UNSUPPORTED elsewhere).
  *     There is no CPU fallback.
  *   - Calls on distinct streams with distinct output/workspace buffers may be
@@ -72,7 +77,7 @@ typedef struct avggt_params {
   int32_t tokens_per_frame;  /* L; must equal n_special + grid_h * grid_w                             */
   int32_t grid_h, grid_w;    /* n_h, n_w: patch grid of one frame                                     */
   int32_t n_special;         /* special tokens per frame (5 for VGGT and pi^3), >= 0                  */
-  int32_t n_heads;           /* H >= 1                                                                */
+  int32_t n_heads;           /* H, 1 <= H <= 32                                                       */
   int32_t head_dim;          /* d; must be 64                                                         */
   int32_t sigma;             /* subsampling factor: 1 (dense), 2, 4, 6, 9 -> (s_h, s_w) =
                                 (1,1), (1,2), (2,2), (2,3), (3,3)  (Sec. 4.3, Subsampling Strategy)   */
@@ -137,7 +142,8 @@ int avggt_build_kv(const avggt_params* p, const void* K, const void* V,
  *     AVGGT_ERR_STATIC_SCRATCH before anything is enqueued;
  *   - the first call on each device looks up the array's device address (and the device's
  *     properties) with that device current; make that first call before any stream capture
- *     begins.  Later calls only enqueue kernels;
+ *     begins.  Later calls only enqueue kernels.  The address is kept for the life of the
+ *     process: after a cudaDeviceReset it is stale and this entry point must not be used again;
  *   - all calls on one device share the one array.  Each call rewrites every element it later
  *     reads, so the previous call's contents do no harm and nothing needs clearing; but two
  *     calls whose kernels overlap on the GPU (different streams, or different host threads)
@@ -163,8 +169,12 @@ int avggt_build_kv_noalloc(const avggt_params* p, const void* K, const void* V,
  *   kmean, vmean  device, float [H, d]; read only when mean_fill != 0 and |D| > 0
  *   O             device, bf16 [N*L, H, d]       written
  *   lse           device, float [N*L, H] or NULL: natural-log normaliser ln(Z) + max-shift
- *   ws            device scratch of at least attn_ws_bytes; the first 16 bytes are a status
- *                 block that the call clears and that avggt_check_status reads.
+ *   ws            device scratch of at least attn_ws_bytes.  It starts with a 256-byte status
+ *                 block that the call clears on the stream and whose first 16 bytes
+ *                 avggt_check_status reads.  The kernel looks at the block when it starts (a
+ *                 launch in which a wait has run out is abandoned by its remaining thread
+ *                 blocks), so one workspace serves one attention launch at a time: launches that
+ *                 may be in flight together need a workspace each.
  */
 int avggt_global_attn(const avggt_params* p, const void* Q, const void* K, const void* V,
                       const void* Kc, const void* Vc, const float* kmean, const float* vmean,
@@ -215,6 +225,43 @@ int avggt_global_attn_shard(const avggt_params* p, int64_t n_kept_total, int64_t
                             const void* Q, const void* K, const void* V,
                             const void* Kc, const void* Vc, const float* kmean, const float* vmean,
                             void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * The exchange step of a frame-sharded run, in two library calls around the caller's two collectives
+ * (Sec. 4.3 defines S and the mean pair over all frames, so the ranks exchange their compact K/V and
+ * the sums behind the mean once per layer; the library itself does no communication).
+ *
+ * avggt_build_kv_shard: avggt_build_kv for this rank's frames (`p` describes them), writing straight
+ * into this rank's slot of the exchange buffer and leaving the mean un-normalised.
+ *   slot        device, bf16 [2][H][slot_rows][d]: compact K, then compact V, head-major; rows
+ *               [M, slot_rows) of every head are left untouched (zero the buffer once: the rows are
+ *               never read as keys, but they travel)
+ *   slot_rows   rows per head in a slot, >= M of this shard (use the largest shard's M on every rank)
+ *   idx         as for avggt_build_kv (token indices local to the shard), may be NULL
+ *   sums        device, float [2][H][d]: sums of K, then of V, over this shard's dropped tokens
+ *               (zero-filled when the shard drops none); may be NULL when mean_fill == 0
+ *   ws          as for avggt_build_kv
+ * The caller then all-gathers the slots into [n_ranks][2][H][slot_rows][d] (in place when `slot`
+ * already lies inside that buffer) and all-reduces `sums`.
+ *
+ * avggt_shard_assemble: the gathered slots -> one compact K/V pair in ascending token order (ranks own
+ * ascending frame ranges), and the mean pair = reduced sums / n_dropped_total.
+ *   gathered         device, bf16 [n_ranks][2][H][slot_rows][d]
+ *   kept             host, int64 [n_ranks]: M of every rank's shard (a pure function of the split)
+ *   sums             device, float [2][H][d], after the all-reduce; read when mean_fill != 0 and
+ *                    n_dropped_total > 0
+ *   Kc, Vc           device, bf16 [H][sum of kept][d]            written
+ *   kmean, vmean     device, float [H][d]                        written (same condition as sums)
+ *   1 <= n_ranks <= 64.  Of `p` the call uses n_heads, head_dim and mean_fill.
+ * Cost of the assembly: one read and one write of the compact K/V (0.57 GB at 800 frames, s = 9).
+ */
+int avggt_build_kv_shard(const avggt_params* p, const void* K, const void* V,
+                         void* slot, int64_t slot_rows, int32_t* idx, float* sums,
+                         void* ws, size_t ws_bytes, void* cuda_stream);
+int avggt_shard_assemble(const avggt_params* p, const void* gathered, int32_t n_ranks,
+                         const int64_t* kept, int64_t slot_rows, const float* sums,
+                         int64_t n_dropped_total, void* Kc, void* Vc,
+                         float* kmean, float* vmean, void* cuda_stream);
 
 /*
  * Frame attention of a converted early global block (Sec. 4.2, "Global-to-Frame Attention

@@ -26,6 +26,7 @@ AVGGT_MEAN_OFF, AVGGT_MEAN_UNIT, AVGGT_MEAN_FILL = 0, 1, 2
 EXPORTS = (
     "avggt_kv_count", "avggt_workspace_bytes", "avggt_build_kv", "avggt_build_kv_noalloc", "avggt_global_attn",
     "avggt_frame_attn", "avggt_build_kv_indexed", "avggt_global_attn_indexed", "avggt_global_attn_shard",
+    "avggt_build_kv_shard", "avggt_shard_assemble",
     "avggt_check_status", "avggt_strerror", "avggt_last_cuda_error", "avggt_version",
 )
 
@@ -91,6 +92,10 @@ def lib():
         L.avggt_global_attn_indexed.restype = ctypes.c_int
         L.avggt_global_attn_shard.argtypes = [pp, ctypes.c_int64, ctypes.c_int64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.avggt_global_attn_shard.restype = ctypes.c_int
+        L.avggt_build_kv_shard.argtypes = [pp, vp, vp, vp, ctypes.c_int64, vp, vp, vp, ctypes.c_size_t, vp]
+        L.avggt_build_kv_shard.restype = ctypes.c_int
+        L.avggt_shard_assemble.argtypes = [pp, vp, ctypes.c_int32, i64p, ctypes.c_int64, vp, ctypes.c_int64, vp, vp, vp, vp, vp]
+        L.avggt_shard_assemble.restype = ctypes.c_int
         L.avggt_check_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
         L.avggt_strerror.argtypes = [ctypes.c_int]
         for f in (L.avggt_kv_count, L.avggt_workspace_bytes, L.avggt_build_kv, L.avggt_global_attn, L.avggt_check_status):
@@ -179,6 +184,22 @@ def avggt_global_attn_shard(params, n_kept_total, n_dropped_total, Q, K, V, Kc, 
     _check(lib().avggt_global_attn_shard(ctypes.byref(params), n_kept_total, n_dropped_total, _ptr(Q), _ptr(K), _ptr(V),
                                          _ptr(Kc), _ptr(Vc), _ptr(kmean), _ptr(vmean), _ptr(O), _ptr(lse), _ptr(ws),
                                          ws_bytes, stream), "avggt_global_attn_shard")
+
+
+def avggt_build_kv_shard(params, K, V, slot, slot_rows, idx, sums, ws, ws_bytes, stream=None):
+    """Enqueue the compaction of one frame shard into its slot [2][H][slot_rows][d] of the exchange buffer;
+    ``sums`` [2][H][d] receives the un-normalised sums over the shard's dropped tokens."""
+    _check(lib().avggt_build_kv_shard(ctypes.byref(params), _ptr(K), _ptr(V), _ptr(slot), slot_rows, _ptr(idx), _ptr(sums),
+                                      _ptr(ws), ws_bytes, stream), "avggt_build_kv_shard")
+
+
+def avggt_shard_assemble(params, gathered, kept, slot_rows, sums, n_dropped_total, Kc, Vc, kmean, vmean, stream=None):
+    """Enqueue the assembly of the gathered slots [n_ranks][2][H][slot_rows][d] into Kc, Vc [H][sum(kept)][d] and
+    the division of the all-reduced sums by the total dropped count.  ``kept``: M of every rank (host ints)."""
+    arr = (ctypes.c_int64 * len(kept))(*[int(k) for k in kept])
+    _check(lib().avggt_shard_assemble(ctypes.byref(params), _ptr(gathered), len(kept), arr, slot_rows, _ptr(sums),
+                                      n_dropped_total, _ptr(Kc), _ptr(Vc), _ptr(kmean), _ptr(vmean), stream),
+           "avggt_shard_assemble")
 
 
 def avggt_frame_attn(params, Q, K, V, O, lse, ws, ws_bytes, stream=None):

@@ -13,17 +13,9 @@ namespace {
 
 thread_local char g_cuda_error[256] = "";
 
-int record_cuda(cudaError_t e) {
-  if (e == cudaSuccess) return AVGGT_OK;
-  std::strncpy(g_cuda_error, cudaGetErrorString(e), sizeof(g_cuda_error) - 1);
-  g_cuda_error[sizeof(g_cuda_error) - 1] = 0;
-  (void)cudaGetLastError();   // clear the sticky-less error state
-  return AVGGT_ERR_CUDA;
-}
-
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-struct DeviceInfo { int sm_count; int cc_major; };
+}  // namespace
 
 // Properties of the current device (queried once per device index).
 int device_info(DeviceInfo* out) {
@@ -48,7 +40,17 @@ int device_info(DeviceInfo* out) {
   return out->cc_major == 10 ? AVGGT_OK : AVGGT_ERR_UNSUPPORTED;
 }
 
-}  // namespace
+int record_message(const char* text) {
+  std::strncpy(g_cuda_error, text, sizeof(g_cuda_error) - 1);
+  g_cuda_error[sizeof(g_cuda_error) - 1] = 0;
+  return AVGGT_ERR_CUDA;
+}
+
+int record_cuda(cudaError_t e) {
+  if (e == cudaSuccess) return AVGGT_OK;
+  (void)cudaGetLastError();   // clear the non-sticky error state
+  return record_message(cudaGetErrorString(e));
+}
 
 int make_plan(const avggt_params* p, Plan* pl) {
   if (p == nullptr || pl == nullptr) return AVGGT_ERR_INVALID_ARG;
@@ -141,32 +143,53 @@ int avggt_build_kv(const avggt_params* p, const void* K, const void* V, void* Kc
   return record_cuda(launch_build_kv(pl, di.sm_count, K, V, Kc, Vc, idx, kmean, vmean, ws, static_cast<cudaStream_t>(cuda_stream)));
 }
 
+// One attention call: which buffers, on which stream.
+struct AttnCall {
+  const void *Q, *K, *V, *Kc, *Vc;
+  const float *kmean, *vmean;
+  void* O;
+  float* lse;
+  void* ws;
+  size_t ws_bytes;
+  void* stream;
+  const int32_t* slot_of_token;   // caller-chosen retained set, else null
+  bool frame_mode;                // frame attention (Sec. 4.2): Kc, Vc, kmean, vmean play no part
+};
+
+// Validation and launch shared by every attention entry point.  Everything that can be rejected on the
+// host is rejected before anything is enqueued.
+static int run_attn(const Plan& pl, const AttnCall& c) {
+  const bool need_diag = !c.frame_mode && pl.diag != 0 && pl.n_dropped > 0;
+  const bool need_mean = !c.frame_mode && pl.mean_fill != 0 && pl.n_dropped > 0;
+  if (!c.Q || !c.O || !c.ws) return AVGGT_ERR_INVALID_ARG;
+  if (c.frame_mode ? (!c.K || !c.V) : (pl.M > 0 && (!c.Kc || !c.Vc))) return AVGGT_ERR_INVALID_ARG;
+  if (need_diag && (!c.K || !c.V)) return AVGGT_ERR_INVALID_ARG;
+  if (need_mean && (!c.kmean || !c.vmean)) return AVGGT_ERR_INVALID_ARG;
+  if (!aligned16(c.Q) || !aligned16(c.K) || !aligned16(c.V) || !aligned16(c.Kc) || !aligned16(c.Vc) || !aligned16(c.O) ||
+      !aligned16(c.ws) || !aligned16(c.kmean) || !aligned16(c.vmean) || (reinterpret_cast<uintptr_t>(c.lse) & 3u) ||
+      (reinterpret_cast<uintptr_t>(c.slot_of_token) & 3u))
+    return AVGGT_ERR_ALIGNMENT;
+  DeviceInfo di;
+  int rc = device_info(&di);
+  if (rc != AVGGT_OK) return rc;
+  if (c.ws_bytes < global_attn_ws_bytes(pl, di.sm_count)) return AVGGT_ERR_WORKSPACE_TOO_SMALL;
+  bool tmap_failed = false;
+  const cudaStream_t st = static_cast<cudaStream_t>(c.stream);
+  const cudaError_t e = c.frame_mode
+      ? launch_frame_attn(pl, c.Q, c.K, c.V, c.O, c.lse, c.ws, st, &tmap_failed)
+      : launch_global_attn(pl, di.sm_count, c.Q, c.K, c.V, c.Kc, c.Vc, c.kmean, c.vmean, c.O, c.lse, c.ws, st,
+                           &tmap_failed, c.slot_of_token);
+  if (tmap_failed) return record_message("cuTensorMapEncodeTiled failed");
+  return record_cuda(e);
+}
+
 int avggt_global_attn(const avggt_params* p, const void* Q, const void* K, const void* V, const void* Kc,
                       const void* Vc, const float* kmean, const float* vmean, void* O, float* lse, void* ws,
                       size_t ws_bytes, void* cuda_stream) {
   Plan pl;
   int rc = make_plan(p, &pl);
   if (rc != AVGGT_OK) return rc;
-  const bool need_diag = pl.diag != 0 && pl.n_dropped > 0;
-  const bool need_mean = pl.mean_fill != 0 && pl.n_dropped > 0;
-  if (!Q || !Kc || !Vc || !O || !ws) return AVGGT_ERR_INVALID_ARG;
-  if (need_diag && (!K || !V)) return AVGGT_ERR_INVALID_ARG;
-  if (need_mean && (!kmean || !vmean)) return AVGGT_ERR_INVALID_ARG;
-  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(Kc) || !aligned16(Vc) || !aligned16(O) ||
-      !aligned16(ws) || !aligned16(kmean) || !aligned16(vmean) || (reinterpret_cast<uintptr_t>(lse) & 3u))
-    return AVGGT_ERR_ALIGNMENT;
-  DeviceInfo di;
-  rc = device_info(&di);
-  if (rc != AVGGT_OK) return rc;
-  if (ws_bytes < global_attn_ws_bytes(pl, di.sm_count)) return AVGGT_ERR_WORKSPACE_TOO_SMALL;
-  bool tmap_failed = false;
-  cudaError_t e = launch_global_attn(pl, di.sm_count, Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws,
-                                     static_cast<cudaStream_t>(cuda_stream), &tmap_failed);
-  if (tmap_failed) {
-    std::strncpy(g_cuda_error, "cuTensorMapEncodeTiled failed", sizeof(g_cuda_error) - 1);
-    return AVGGT_ERR_CUDA;
-  }
-  return record_cuda(e);
+  return run_attn(pl, AttnCall{Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws, ws_bytes, cuda_stream, nullptr, false});
 }
 
 // Plan of a problem whose retained set is a caller-supplied list of n_kept tokens.
@@ -186,7 +209,8 @@ int avggt_build_kv_indexed(const avggt_params* p, const int32_t* idx, int64_t n_
   Plan pl;
   int rc = make_indexed_plan(p, n_kept, &pl);
   if (rc != AVGGT_OK) return rc;
-  if (!idx || !slot_of_token || !K || !V || !Kc || !Vc || !ws) return AVGGT_ERR_INVALID_ARG;
+  if (!slot_of_token || !K || !V || !ws) return AVGGT_ERR_INVALID_ARG;
+  if (n_kept > 0 && (!idx || !Kc || !Vc)) return AVGGT_ERR_INVALID_ARG;
   if (pl.mean_fill != 0 && (!kmean || !vmean)) return AVGGT_ERR_INVALID_ARG;
   if (!aligned16(K) || !aligned16(V) || !aligned16(Kc) || !aligned16(Vc) || !aligned16(ws) ||
       (reinterpret_cast<uintptr_t>(idx) & 3u) || (reinterpret_cast<uintptr_t>(slot_of_token) & 3u) ||
@@ -206,27 +230,8 @@ int avggt_global_attn_indexed(const avggt_params* p, int64_t n_kept, const int32
   Plan pl;
   int rc = make_indexed_plan(p, n_kept, &pl);
   if (rc != AVGGT_OK) return rc;
-  const bool need_diag = pl.diag != 0 && pl.n_dropped > 0;
-  const bool need_mean = pl.mean_fill != 0 && pl.n_dropped > 0;
-  if (!Q || !Kc || !Vc || !O || !ws || !slot_of_token) return AVGGT_ERR_INVALID_ARG;
-  if (need_diag && (!K || !V)) return AVGGT_ERR_INVALID_ARG;
-  if (need_mean && (!kmean || !vmean)) return AVGGT_ERR_INVALID_ARG;
-  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(Kc) || !aligned16(Vc) || !aligned16(O) ||
-      !aligned16(ws) || !aligned16(kmean) || !aligned16(vmean) || (reinterpret_cast<uintptr_t>(lse) & 3u) ||
-      (reinterpret_cast<uintptr_t>(slot_of_token) & 3u))
-    return AVGGT_ERR_ALIGNMENT;
-  DeviceInfo di;
-  rc = device_info(&di);
-  if (rc != AVGGT_OK) return rc;
-  if (ws_bytes < global_attn_ws_bytes(pl, di.sm_count)) return AVGGT_ERR_WORKSPACE_TOO_SMALL;
-  bool tmap_failed = false;
-  cudaError_t e = launch_global_attn(pl, di.sm_count, Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws,
-                                     static_cast<cudaStream_t>(cuda_stream), &tmap_failed, slot_of_token);
-  if (tmap_failed) {
-    std::strncpy(g_cuda_error, "cuTensorMapEncodeTiled failed", sizeof(g_cuda_error) - 1);
-    return AVGGT_ERR_CUDA;
-  }
-  return record_cuda(e);
+  if (!slot_of_token) return AVGGT_ERR_INVALID_ARG;
+  return run_attn(pl, AttnCall{Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws, ws_bytes, cuda_stream, slot_of_token, false});
 }
 
 int avggt_global_attn_shard(const avggt_params* p, int64_t n_kept_total, int64_t n_dropped_total, const void* Q,
@@ -239,26 +244,50 @@ int avggt_global_attn_shard(const avggt_params* p, int64_t n_kept_total, int64_t
   if (n_kept_total < pl.M || n_dropped_total < pl.n_dropped) return AVGGT_ERR_INVALID_ARG;
   pl.M = n_kept_total;
   pl.n_dropped = n_dropped_total;
-  const bool need_diag = pl.diag != 0 && pl.n_dropped > 0;
-  const bool need_mean = pl.mean_fill != 0 && pl.n_dropped > 0;
-  if (!Q || !Kc || !Vc || !O || !ws) return AVGGT_ERR_INVALID_ARG;
-  if (need_diag && (!K || !V)) return AVGGT_ERR_INVALID_ARG;
-  if (need_mean && (!kmean || !vmean)) return AVGGT_ERR_INVALID_ARG;
-  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(Kc) || !aligned16(Vc) || !aligned16(O) ||
-      !aligned16(ws) || !aligned16(kmean) || !aligned16(vmean) || (reinterpret_cast<uintptr_t>(lse) & 3u))
+  return run_attn(pl, AttnCall{Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws, ws_bytes, cuda_stream, nullptr, false});
+}
+
+int avggt_build_kv_shard(const avggt_params* p, const void* K, const void* V, void* slot, int64_t slot_rows,
+                         int32_t* idx, float* sums, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Plan pl;
+  int rc = make_plan(p, &pl);
+  if (rc != AVGGT_OK) return rc;
+  if (!K || !V || !slot || !ws) return AVGGT_ERR_INVALID_ARG;
+  if (slot_rows < pl.M) return AVGGT_ERR_INVALID_ARG;
+  if (pl.mean_fill != 0 && !sums) return AVGGT_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(V) || !aligned16(slot) || !aligned16(ws) || (reinterpret_cast<uintptr_t>(idx) & 3u) ||
+      !aligned16(sums))
     return AVGGT_ERR_ALIGNMENT;
   DeviceInfo di;
   rc = device_info(&di);
   if (rc != AVGGT_OK) return rc;
-  if (ws_bytes < global_attn_ws_bytes(pl, di.sm_count)) return AVGGT_ERR_WORKSPACE_TOO_SMALL;
-  bool tmap_failed = false;
-  cudaError_t e = launch_global_attn(pl, di.sm_count, Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws,
-                                     static_cast<cudaStream_t>(cuda_stream), &tmap_failed);
-  if (tmap_failed) {
-    std::strncpy(g_cuda_error, "cuTensorMapEncodeTiled failed", sizeof(g_cuda_error) - 1);
-    return AVGGT_ERR_CUDA;
-  }
-  return record_cuda(e);
+  if (ws_bytes < build_kv_ws_bytes(pl, di.sm_count)) return AVGGT_ERR_WORKSPACE_TOO_SMALL;
+  const size_t part = static_cast<size_t>(pl.H) * static_cast<size_t>(slot_rows) * pl.d;   // elements of the K part of a slot
+  void* Vc = static_cast<char*>(slot) + part * 2;
+  float* vsum = sums ? sums + static_cast<size_t>(pl.H) * pl.d : nullptr;
+  return record_cuda(launch_build_kv(pl, di.sm_count, K, V, slot, Vc, idx, sums, vsum, ws,
+                                     static_cast<cudaStream_t>(cuda_stream), nullptr, nullptr, slot_rows, true));
+}
+
+int avggt_shard_assemble(const avggt_params* p, const void* gathered, int32_t n_ranks, const int64_t* kept,
+                         int64_t slot_rows, const float* sums, int64_t n_dropped_total, void* Kc, void* Vc,
+                         float* kmean, float* vmean, void* cuda_stream) {
+  Plan pl;
+  int rc = make_plan(p, &pl);
+  if (rc != AVGGT_OK) return rc;
+  if (!gathered || !kept || !Kc || !Vc || n_ranks < 1 || n_ranks > kMaxShardRanks || n_dropped_total < 0)
+    return AVGGT_ERR_INVALID_ARG;
+  for (int r = 0; r < n_ranks; ++r)
+    if (kept[r] < 0 || kept[r] > slot_rows) return AVGGT_ERR_INVALID_ARG;
+  const bool need_mean = pl.mean_fill != 0 && n_dropped_total > 0;
+  if (need_mean && (!sums || !kmean || !vmean)) return AVGGT_ERR_INVALID_ARG;
+  if (!aligned16(gathered) || !aligned16(Kc) || !aligned16(Vc) || !aligned16(sums) || !aligned16(kmean) || !aligned16(vmean))
+    return AVGGT_ERR_ALIGNMENT;
+  DeviceInfo di;
+  rc = device_info(&di);
+  if (rc != AVGGT_OK) return rc;
+  return record_cuda(launch_assemble_shards(gathered, n_ranks, kept, pl.H, pl.d, slot_rows, Kc, Vc, need_mean ? sums : nullptr,
+                                            n_dropped_total, kmean, vmean, static_cast<cudaStream_t>(cuda_stream)));
 }
 
 int avggt_frame_attn(const avggt_params* p, const void* Q, const void* K, const void* V, void* O, float* lse, void* ws,
@@ -266,22 +295,8 @@ int avggt_frame_attn(const avggt_params* p, const void* Q, const void* K, const 
   Plan pl;
   int rc = make_plan(p, &pl);
   if (rc != AVGGT_OK) return rc;
-  if (!Q || !K || !V || !O || !ws) return AVGGT_ERR_INVALID_ARG;
-  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(ws) ||
-      (reinterpret_cast<uintptr_t>(lse) & 3u))
-    return AVGGT_ERR_ALIGNMENT;
   if (pl.n_frames > 65535) return AVGGT_ERR_UNSUPPORTED;
-  DeviceInfo di;
-  rc = device_info(&di);
-  if (rc != AVGGT_OK) return rc;
-  if (ws_bytes < global_attn_ws_bytes(pl, di.sm_count)) return AVGGT_ERR_WORKSPACE_TOO_SMALL;
-  bool tmap_failed = false;
-  cudaError_t e = launch_frame_attn(pl, Q, K, V, O, lse, ws, static_cast<cudaStream_t>(cuda_stream), &tmap_failed);
-  if (tmap_failed) {
-    std::strncpy(g_cuda_error, "cuTensorMapEncodeTiled failed", sizeof(g_cuda_error) - 1);
-    return AVGGT_ERR_CUDA;
-  }
-  return record_cuda(e);
+  return run_attn(pl, AttnCall{Q, K, V, nullptr, nullptr, nullptr, nullptr, O, lse, ws, ws_bytes, cuda_stream, nullptr, true});
 }
 
 int avggt_check_status(const void* attn_ws, uint32_t* detail) {

@@ -39,11 +39,13 @@ __device__ __forceinline__ void add_bf16x8(float (&acc)[8], const uint4& v) {
 }
 
 // PASSES = ceil(H * 8 / 32): 16-byte chunks of one row handled per lane.
+// kc_rows: rows per head of the compact arrays (M, or more when the caller's arrays are a slot of a
+// larger exchange buffer).
 template <int PASSES>
 __global__ void __launch_bounds__(kBuildThreads)
 build_kv_kernel(const Plan pl, const uint4* __restrict__ K, const uint4* __restrict__ V, uint4* __restrict__ Kc,
-                uint4* __restrict__ Vc, int32_t* __restrict__ idx, float* __restrict__ partials, const int do_mean,
-                const int32_t* __restrict__ slot_of_token) {
+                uint4* __restrict__ Vc, const int64_t kc_rows, int32_t* __restrict__ idx, float* __restrict__ partials,
+                const int do_mean, const int32_t* __restrict__ slot_of_token) {
   extern __shared__ float red[];   // [kBuildWarps][PASSES * 256]
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
@@ -80,7 +82,7 @@ build_kv_kernel(const Plan pl, const uint4* __restrict__ K, const uint4* __restr
       for (int p = 0; p < PASSES; ++p) {
         const uint32_t c = p * 32 + lane;
         if (c < chunks_per_row) {
-          const size_t dst = (static_cast<size_t>(c >> 3) * static_cast<size_t>(pl.M) + static_cast<size_t>(m)) * 8u + (c & 7u);
+          const size_t dst = (static_cast<size_t>(c >> 3) * static_cast<size_t>(kc_rows) + static_cast<size_t>(m)) * 8u + (c & 7u);
           Kc[dst] = kv[p];
           Vc[dst] = vv[p];
         }
@@ -153,20 +155,71 @@ __global__ void scatter_slots_kernel(const int32_t* __restrict__ idx, int64_t M,
 }
 
 template <int PASSES>
-cudaError_t launch_build(const Plan& pl, int grid, const void* K, const void* V, void* Kc, void* Vc, int32_t* idx,
-                         float* partials, int do_mean, const int32_t* slot_of_token, cudaStream_t st) {
+cudaError_t launch_build(const Plan& pl, int grid, const void* K, const void* V, void* Kc, void* Vc, int64_t kc_rows,
+                         int32_t* idx, float* partials, int do_mean, const int32_t* slot_of_token, cudaStream_t st) {
   const size_t smem = do_mean ? static_cast<size_t>(kBuildWarps) * PASSES * 256 * sizeof(float) : 0;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(build_kv_kernel<PASSES>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
   }
   build_kv_kernel<PASSES><<<grid, kBuildThreads, smem, st>>>(pl, static_cast<const uint4*>(K), static_cast<const uint4*>(V),
-                                                           static_cast<uint4*>(Kc), static_cast<uint4*>(Vc), idx, partials, do_mean,
-                                                           slot_of_token);
+                                                           static_cast<uint4*>(Kc), static_cast<uint4*>(Vc), kc_rows, idx, partials,
+                                                           do_mean, slot_of_token);
   return cudaGetLastError();
 }
 
+// Exchange buffer [n_ranks][2][H][slot_rows][d] (every rank's compact K then V, padded to slot_rows rows per
+// head) -> Kc, Vc [H][M_total][d] with the ranks' rows one after the other.  One thread per 16-byte chunk.
+struct ShardOffsets {
+  int32_t n_ranks;
+  int64_t first[kMaxShardRanks + 1];   // first compact row of rank r; first[n_ranks] = M_total
+};
+__global__ void __launch_bounds__(256)
+assemble_shards_kernel(const uint4* __restrict__ gathered, const ShardOffsets off, const int H, const int64_t slot_rows,
+                       uint4* __restrict__ Kc, uint4* __restrict__ Vc) {
+  const int64_t m_total = off.first[off.n_ranks];
+  const int64_t chunks = 2 * static_cast<int64_t>(H) * m_total * 8;   // 8 chunks of 16 bytes per row of 64 bf16
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < chunks;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int64_t c = i & 7;
+    int64_t row = i >> 3;                       // (which, head, m)
+    const int64_t m = row % m_total;
+    row /= m_total;
+    const int64_t h = row % H;
+    const int64_t which = row / H;
+    int r = 0;
+    while (r + 1 < off.n_ranks && m >= off.first[r + 1]) ++r;
+    const int64_t src = ((((static_cast<int64_t>(r) * 2 + which) * H + h) * slot_rows) + (m - off.first[r])) * 8 + c;
+    const uint4 v = gathered[src];
+    (which == 0 ? Kc : Vc)[(h * m_total + m) * 8 + c] = v;
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_assemble_shards(const void* gathered, int n_ranks, const int64_t* kept, int H, int d, int64_t slot_rows,
+                                   void* Kc, void* Vc, const float* sums, int64_t n_dropped_total, float* kmean,
+                                   float* vmean, cudaStream_t st) {
+  ShardOffsets off;
+  off.n_ranks = n_ranks;
+  off.first[0] = 0;
+  for (int r = 0; r < n_ranks; ++r) off.first[r + 1] = off.first[r] + kept[r];
+  const int64_t chunks = 2 * static_cast<int64_t>(H) * off.first[n_ranks] * 8;
+  if (chunks > 0) {
+    int64_t blocks = (chunks + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    assemble_shards_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(static_cast<const uint4*>(gathered), off, H, slot_rows,
+                                                                         static_cast<uint4*>(Kc), static_cast<uint4*>(Vc));
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  if (sums != nullptr && n_dropped_total > 0) {
+    const int cols2 = 2 * H * d;
+    mean_finalize_kernel<<<(cols2 + 31) / 32, 1024, 0, st>>>(sums, 1, cols2, 1.0f / static_cast<float>(n_dropped_total), kmean, vmean);
+    return cudaGetLastError();
+  }
+  return cudaSuccess;
+}
 
 int build_kv_grid(const Plan& pl, int sm_count) {
   const int64_t by_rows = (pl.n_tok + kBuildWarps - 1) / kBuildWarps;
@@ -182,7 +235,8 @@ size_t build_kv_ws_bytes(const Plan& pl, int sm_count) {
 
 cudaError_t launch_build_kv(const Plan& pl, int sm_count, const void* K, const void* V, void* Kc, void* Vc,
                             int32_t* idx, float* kmean, float* vmean, void* ws, cudaStream_t st,
-                            const int32_t* caller_idx, int32_t* slot_of_token) {
+                            const int32_t* caller_idx, int32_t* slot_of_token, int64_t kc_rows, bool sums_only) {
+  if (kc_rows <= 0) kc_rows = pl.M;
   if (caller_idx != nullptr) {
     // caller-chosen retained set: build the token -> compact position map first
     fill_slots_kernel<<<static_cast<unsigned>((pl.n_tok + 255) / 256), 256, 0, st>>>(slot_of_token, pl.n_tok);
@@ -197,21 +251,22 @@ cudaError_t launch_build_kv(const Plan& pl, int sm_count, const void* K, const v
   const int passes = (pl.H * 8 + 31) / 32;
   cudaError_t e;
   switch (passes) {
-    case 1: e = launch_build<1>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, slot_of_token, st); break;
-    case 2: e = launch_build<2>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, slot_of_token, st); break;
-    case 3: e = launch_build<3>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, slot_of_token, st); break;
-    case 4: e = launch_build<4>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, slot_of_token, st); break;
-    case 5: e = launch_build<5>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, slot_of_token, st); break;
-    case 6: e = launch_build<6>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, slot_of_token, st); break;
-    case 7: e = launch_build<7>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, slot_of_token, st); break;
-    case 8: e = launch_build<8>(pl, grid, K, V, Kc, Vc, idx, partials, do_mean, slot_of_token, st); break;
+    case 1: e = launch_build<1>(pl, grid, K, V, Kc, Vc, kc_rows, idx, partials, do_mean, slot_of_token, st); break;
+    case 2: e = launch_build<2>(pl, grid, K, V, Kc, Vc, kc_rows, idx, partials, do_mean, slot_of_token, st); break;
+    case 3: e = launch_build<3>(pl, grid, K, V, Kc, Vc, kc_rows, idx, partials, do_mean, slot_of_token, st); break;
+    case 4: e = launch_build<4>(pl, grid, K, V, Kc, Vc, kc_rows, idx, partials, do_mean, slot_of_token, st); break;
+    case 5: e = launch_build<5>(pl, grid, K, V, Kc, Vc, kc_rows, idx, partials, do_mean, slot_of_token, st); break;
+    case 6: e = launch_build<6>(pl, grid, K, V, Kc, Vc, kc_rows, idx, partials, do_mean, slot_of_token, st); break;
+    case 7: e = launch_build<7>(pl, grid, K, V, Kc, Vc, kc_rows, idx, partials, do_mean, slot_of_token, st); break;
+    case 8: e = launch_build<8>(pl, grid, K, V, Kc, Vc, kc_rows, idx, partials, do_mean, slot_of_token, st); break;
     default: return cudaErrorInvalidValue;
   }
   if (e != cudaSuccess) return e;
   if (pl.mean_fill != 0) {
     const int cols2 = 2 * pl.H * pl.d;
     if (do_mean) {
-      mean_finalize_kernel<<<(cols2 + 31) / 32, 1024, 0, st>>>(partials, grid, cols2, 1.0f / static_cast<float>(pl.n_dropped), kmean, vmean);
+      const float inv_count = sums_only ? 1.0f : 1.0f / static_cast<float>(pl.n_dropped);
+      mean_finalize_kernel<<<(cols2 + 31) / 32, 1024, 0, st>>>(partials, grid, cols2, inv_count, kmean, vmean);
       e = cudaGetLastError();
     } else {
       e = cudaMemsetAsync(kmean, 0, static_cast<size_t>(pl.H) * pl.d * sizeof(float), st);

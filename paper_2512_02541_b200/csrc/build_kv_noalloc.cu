@@ -20,7 +20,7 @@ namespace {
 
 // Capacity: partial rows of 2 * H * d floats, one per thread block of the compaction kernel.
 constexpr int kStaticMaxCols2 = 2 * 16 * 64;   // H * d <= 1024
-constexpr int kStaticMaxBlocks = 296;          // two blocks per SM on a 148-SM part
+constexpr int kStaticMaxBlocks = 296;          // four blocks per SM on up to 74 SMs' worth of grid (see the entry point)
 constexpr size_t kStaticScratchBytes = static_cast<size_t>(kStaticMaxBlocks) * kStaticMaxCols2 * sizeof(float);
 
 // In host code this name is only a handle for the runtime's symbol lookup, not a device
@@ -30,30 +30,26 @@ static __device__ __align__(256) float g_static_scratch[static_cast<size_t>(kSta
 struct PerDevice {
   bool ready = false;
   void* scratch = nullptr;   // device address of g_static_scratch on this device
-  int sm_count = 0;
-  int cc_major = 0;
 };
 
 std::mutex g_mu;
 PerDevice g_dev[64];
 
-// First call on a device: look up the array's address on that device (which must be the
-// current one) and the device properties.  Nothing here allocates.
-int setup_current_device(PerDevice** out, cudaError_t* cuda_err) {
+// First call on a device: look up the array's address on that device, which must be the
+// current one and an sm_100 part (the caller has checked).  Nothing here allocates.  The address
+// is kept for the life of the process; a cudaDeviceReset invalidates it.
+int setup_current_device(PerDevice** out) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) { *cuda_err = e; return AVGGT_ERR_CUDA; }
+  if (e != cudaSuccess) return record_cuda(e);
   if (dev < 0 || dev >= 64) return AVGGT_ERR_UNSUPPORTED;
   std::lock_guard<std::mutex> lock(g_mu);
   PerDevice& pd = g_dev[dev];
   if (!pd.ready) {
     void* ptr = nullptr;
     e = cudaGetSymbolAddress(&ptr, g_static_scratch);
-    if (e != cudaSuccess || ptr == nullptr) { *cuda_err = e; return AVGGT_ERR_CUDA; }
-    e = cudaDeviceGetAttribute(&pd.sm_count, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) { *cuda_err = e; return AVGGT_ERR_CUDA; }
-    e = cudaDeviceGetAttribute(&pd.cc_major, cudaDevAttrComputeCapabilityMajor, dev);
-    if (e != cudaSuccess) { *cuda_err = e; return AVGGT_ERR_CUDA; }
+    if (e != cudaSuccess) return record_cuda(e);
+    if (ptr == nullptr) return record_message("cudaGetSymbolAddress returned a null address");
     pd.scratch = ptr;
     pd.ready = true;
   }
@@ -80,17 +76,19 @@ extern "C" int avggt_build_kv_noalloc(const avggt_params* p, const void* K, cons
     return AVGGT_ERR_ALIGNMENT;
   // the fixed array holds rows of at most kStaticMaxCols2 floats
   if (2 * pl.H * pl.d > kStaticMaxCols2) return AVGGT_ERR_STATIC_SCRATCH;
-  PerDevice* pd = nullptr;
-  cudaError_t ce = cudaSuccess;
-  rc = setup_current_device(&pd, &ce);
+  // the device is checked before the symbol lookup: on another architecture the library holds no
+  // image of the array and the lookup itself would fail with an unrelated CUDA error
+  DeviceInfo di;
+  rc = device_info(&di);
   if (rc != AVGGT_OK) return rc;
-  if (pd->cc_major != 10) return AVGGT_ERR_UNSUPPORTED;
+  PerDevice* pd = nullptr;
+  rc = setup_current_device(&pd);
+  if (rc != AVGGT_OK) return rc;
   // The compaction kernel runs four blocks per SM it is told about; telling it about fewer SMs
   // keeps its partial rows within the fixed array.
-  int sm_eff = pd->sm_count;
+  int sm_eff = di.sm_count;
   if (sm_eff > kStaticMaxBlocks / 4) sm_eff = kStaticMaxBlocks / 4;
   if (build_kv_ws_bytes(pl, sm_eff) > kStaticScratchBytes) return AVGGT_ERR_STATIC_SCRATCH;
-  ce = launch_build_kv(pl, sm_eff, K, V, Kc, Vc, idx, kmean, vmean, pd->scratch, static_cast<cudaStream_t>(cuda_stream));
-  if (ce != cudaSuccess) { (void)cudaGetLastError(); return AVGGT_ERR_CUDA; }
-  return AVGGT_OK;
+  return record_cuda(launch_build_kv(pl, sm_eff, K, V, Kc, Vc, idx, kmean, vmean, pd->scratch,
+                                     static_cast<cudaStream_t>(cuda_stream)));
 }

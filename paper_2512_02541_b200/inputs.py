@@ -76,25 +76,29 @@ WORKLOADS = {
 }
 
 
-def make_qkv(wl, seed=0, device="cpu", frames_per_chunk=16):
+def make_qkv(wl, seed=0, device="cpu", frames_per_chunk=16, frame_range=None):
     """Return (Q, K, V), each a bf16 tensor [N*L, H, d] on ``device``.
 
     The generator is seeded per call; CPU and CUDA generators give different
     streams, so a parity test draws once and hands the same tensors (copied to
-    the host) to the oracle.
+    the host) to the oracle.  ``frame_range = (f0, f1)`` returns only the rows
+    of frames [f0, f1) of the very same tensors (all frames are still drawn, so
+    every rank of a frame-sharded run sees its part of one common problem).
     """
     gen = torch.Generator(device=device)
     gen.manual_seed(seed)
     L, H, d = wl.tokens_per_frame, wl.n_heads, wl.head_dim
     n_tok = wl.n_tokens
     shape = (n_tok, H, d)
+    k0, k1 = (0, wl.n_frames) if frame_range is None else frame_range
     if wl.recipe == "iid":
         Q = torch.randn(shape, generator=gen, device=device, dtype=torch.float32) * 3.0
         K = torch.randn(shape, generator=gen, device=device, dtype=torch.float32)
         V = torch.randn(shape, generator=gen, device=device, dtype=torch.float32)
-        return Q.bfloat16(), K.bfloat16(), V.bfloat16()
+        return tuple(t[k0 * L:k1 * L].bfloat16().contiguous() for t in (Q, K, V))
     if wl.recipe != "proj":
         raise ValueError(f"unknown recipe {wl.recipe!r}")
+    shape = ((k1 - k0) * L, H, d)
 
     C = H * d
     w_q = torch.randn((C, C), generator=gen, device=device, dtype=torch.float32) * (C ** -0.5)
@@ -107,31 +111,40 @@ def make_qkv(wl, seed=0, device="cpu", frames_per_chunk=16):
         nf = min(frames_per_chunk, wl.n_frames - f0)
         x = torch.randn((nf, L, C), generator=gen, device=device, dtype=torch.float32)
         x[:, wl.n_special:, :] += 0.5 * shared
-        x = x.reshape(nf * L, C)
-        qk = (x @ w_q).bfloat16().reshape(nf * L, H, d)
-        Q[f0 * L:(f0 + nf) * L] = qk
-        K[f0 * L:(f0 + nf) * L] = qk
-        V[f0 * L:(f0 + nf) * L] = (x @ w_v).bfloat16().reshape(nf * L, H, d)
+        a, b = max(f0, k0), min(f0 + nf, k1)          # frames of this chunk that the caller keeps
+        if a >= b:
+            continue
+        x = x[a - f0:b - f0].reshape((b - a) * L, C)
+        qk = (x @ w_q).bfloat16().reshape((b - a) * L, H, d)
+        Q[(a - k0) * L:(b - k0) * L] = qk
+        K[(a - k0) * L:(b - k0) * L] = qk
+        V[(a - k0) * L:(b - k0) * L] = (x @ w_v).bfloat16().reshape((b - a) * L, H, d)
     return Q, K, V
 
 
-def sample_rows(wl, n_rows, seed=0, tile=128):
+def sample_rows(wl, n_rows, seed=0, tile=128, must_include=()):
     """A fixed, stratified sample of query rows for parity checks on workloads
     too large for the oracle to cover in full: the first and last rows, the
     special tokens of the first and last frame, rows on both sides of tile
-    boundaries, the ragged tail tile, and uniformly random rows.
+    boundaries at the start, in the middle and at the end of the sequence (every
+    position class of a row within a pair of tiles: row mod 2*tile in
+    {0, tile-1, tile, 2*tile-1}), the ragged tail tile, the rows the caller
+    names in ``must_include``, and uniformly random rows up to ``n_rows``.
     """
     n_tok, L = wl.n_tokens, wl.tokens_per_frame
     if n_rows >= n_tok:
         return torch.arange(n_tok)
-    picks = set()
+    picks = set(int(r) for r in must_include)
     picks.update(range(min(wl.n_special + 3, n_tok)))                      # frame 0 specials + first patches
     picks.update(range((wl.n_frames - 1) * L, (wl.n_frames - 1) * L + wl.n_special + 3))
     picks.update(range(max(0, n_tok - 4), n_tok))                          # very last rows
     tail0 = (n_tok // tile) * tile
     picks.update(range(max(0, tail0 - 2), min(n_tok, tail0 + 2)))          # around the tail tile
-    for b in (1, 2, n_tok // (2 * tile)):
-        picks.update(range(max(0, b * tile - 2), min(n_tok, b * tile + 2)))
+    pair = 2 * tile
+    n_pairs = max(1, n_tok // pair)
+    for b in sorted({0, 1, n_pairs // 3, n_pairs // 2, (2 * n_pairs) // 3, max(0, n_pairs - 2), n_pairs - 1}):
+        for off in (0, 1, tile - 1, tile, tile + 1, pair - 1):
+            picks.add(b * pair + off)
     picks = {p for p in picks if 0 <= p < n_tok}
     gen = torch.Generator()
     gen.manual_seed(seed)

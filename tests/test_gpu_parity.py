@@ -59,6 +59,24 @@ def _check_build(ocfg, layer, K, V):
     return Kh, Vh
 
 
+def _stratified_rows(wl, ocfg, n_rows):
+    """Sample of query rows for the full-size checks: ``inputs.sample_rows`` (sequence ends, tile-boundary
+    classes, tail, random rows) plus, for the first, the last and five frames in between, one special
+    token, one retained patch and one dropped patch, so that every kind of row (and with it every
+    combination of the diagonal and mean terms) is met in frame 0 and well inside the sequence."""
+    L = wl.tokens_per_frame
+    rng = np.random.default_rng(5)
+    frames = sorted({0, wl.n_frames - 1, *rng.integers(0, wl.n_frames, 5).tolist(), wl.n_frames // 2})
+    must = []
+    for f in frames:
+        kept = orc.kept_slot_mask(ocfg, f)
+        special = np.arange(L) < wl.n_special
+        for members in (np.flatnonzero(special), np.flatnonzero(kept & ~special), np.flatnonzero(~kept)):
+            if len(members):
+                must.append(f * L + int(rng.choice(members)))
+    return inputs.sample_rows(wl, n_rows, must_include=must).numpy()
+
+
 def _check_attn(ocfg, Q, Kh, Vh, O, rows=None, lse=None):
     Qh = _host(Q)
     if rows is None:
@@ -141,32 +159,41 @@ def test_large_logits_and_dominant_diagonal():
 
 
 def test_vggt_100_frames_sampled_rows():
-    """The benchmark workload (100 frames, 37x37 grid, s=4) in the launch configuration
-    bench.py times, checked on a stratified sample of rows the oracle computes one by one."""
+    """The 100-frame benchmark configuration (37x37 grid, s=4) in the launch configuration
+    bench.py times, checked on a stratified sample of 2048 rows (the oracle's blocked form:
+    one matrix product per head over the sampled rows, the arithmetic per row unchanged)."""
     wl = inputs.WORKLOADS["vggt_n100_s4"]
     params, ocfg, layer, Q, K, V, O = _run_gpu(wl)
     assert (layer.M, layer.n_dropped) == (36600, 100800)
     Kh, Vh = _check_build(ocfg, layer, K, V)
-    rows = inputs.sample_rows(wl, 512).numpy()
+    rows = _stratified_rows(wl, ocfg, 2048)
     _check_attn(ocfg, Q, Kh, Vh, O, rows=rows)
+    # a handful of the same rows through the oracle's row-by-row form as well
+    few = rows[:: max(1, len(rows) // 12)]
+    want = orc.global_attn(ocfg, _host(Q), Kh, Vh, rows=few)
+    got = O[torch.as_tensor(few, device=O.device)].float().cpu().numpy().astype(np.float64)
+    assert np.abs(got - want).max() <= MAX_ABS_TOL
     # properties that hold at any size: every row written and finite
     assert torch.isfinite(O.float()).all()
 
 
 @pytest.mark.parametrize("name,n_rows", [
-    ("vggt_n300_s6", 96),     # 412,200 queries x 75,600 compact keys
-    ("vggt_n800_s9", 64),     # 1,099,200 queries x 139,200 compact keys: the long-context case
-    ("vggt_n333_s1", 48),     # dense layer (both switches off), 457,542 x 457,542
-    ("vggt_n333_s9", 64),     # the other end of the factor sweep
+    ("vggt_n300_s6", 512),    # 412,200 queries x 75,600 compact keys
+    ("vggt_n800_s9", 512),    # 1,099,200 queries x 139,200 compact keys: the long-context case bench.py times
+    ("vggt_n333_s1", 160),    # dense layer (both switches off), 457,542 x 457,542
+    ("vggt_n333_s2", 256),    # the factor sweep at 333 frames
+    ("vggt_n333_s4", 512),
+    ("vggt_n333_s6", 512),
+    ("vggt_n333_s9", 512),
 ])
 def test_full_size_configs_sampled_rows(name, n_rows):
-    """The larger benchmark configurations at full size, in the launch configuration bench.py times:
-    compaction checked in full against the oracle, attention on a stratified sample of rows the
-    oracle computes one by one, and every output row finite."""
+    """Every larger benchmark configuration at full size, in the launch configuration bench.py times:
+    compaction checked in full against the oracle, attention on a stratified sample of rows
+    (the oracle's blocked form over the sample), and every output row finite."""
     wl = inputs.WORKLOADS[name]
     params, ocfg, layer, Q, K, V, O = _run_gpu(wl)
     Kh, Vh = _check_build(ocfg, layer, K, V)
-    rows = inputs.sample_rows(wl, n_rows).numpy()
+    rows = _stratified_rows(wl, ocfg, n_rows)
     _check_attn(ocfg, Q, Kh, Vh, O, rows=rows)
     assert torch.isfinite(O.float()).all()
     del Q, K, V, O, layer

@@ -1,7 +1,8 @@
-"""Frame-sharded layer on one GPU: the shards of a two-rank split are computed one after the other
-(no kernel waits on another), their compact K/V and mean pairs are combined as the exchange step
-combines them, and every shard's output is checked against the fp64 oracle of the whole sequence.
-The collectives themselves are covered by the two-rank gloo test on the CPU."""
+"""Frame-sharded layer on one GPU: the shards of a two- or three-rank split are computed one after the
+other (no kernel waits on another) through the entry points a rank calls (`avggt_build_kv_shard`,
+`avggt_shard_assemble`, `avggt_global_attn_shard`), and every shard's output is checked against the
+fp64 oracle of the whole sequence.  The collectives themselves are covered by the two-rank gloo test
+on the CPU."""
 
 import socket
 
@@ -18,7 +19,9 @@ pytestmark = pytest.mark.gpu
 
 
 def _shard_run(wl, world, keep_first=False, seed=0):
-    """Returns (Q, K, V, O) of the whole sequence, O assembled from `world` sequentially computed shards."""
+    """Returns (Q, K, V, O, Kc, Vc, kmean, vmean) of the whole sequence, O assembled from `world` sequentially
+    computed shards.  The all-gather is stood in for by every shard writing its own slot of one common exchange
+    buffer, the all-reduce by adding the shards' sums."""
     Q, K, V = inputs.make_qkv(wl, seed=seed, device="cuda")
     L, H, d = wl.tokens_per_frame, wl.n_heads, wl.head_dim
     mk = lambda n, kff: P.make_params(n, wl.grid_h, wl.grid_w, wl.n_special, H, d, wl.sigma, diag=wl.diag,
@@ -27,21 +30,21 @@ def _shard_run(wl, world, keep_first=False, seed=0):
     params = [mk(f1 - f0, keep_first and r == 0) for r, (f0, f1) in enumerate(ranges)]
     counts = [P.avggt_kv_count(p) for p in params]
     kept, dropped = [c[0] for c in counts], [c[1] for c in counts]
-    locals_ = []
+    slot_rows = max(kept)
+    gathered = torch.zeros((world, 2, H, slot_rows, d), dtype=torch.bfloat16, device="cuda")
+    total = torch.zeros((2, H, d), device="cuda")
     for r, (f0, f1) in enumerate(ranges):
         bws, _ = P.avggt_workspace_bytes(params[r])
-        Kc = torch.empty((H, kept[r], d), dtype=torch.bfloat16, device="cuda"); Vc = torch.empty_like(Kc)
-        km = torch.zeros((H, d), device="cuda"); vm = torch.zeros_like(km)
+        sums = torch.full((2, H, d), float("nan"), device="cuda")
         ws = torch.empty((max(bws, 16),), dtype=torch.uint8, device="cuda")
-        P.avggt_build_kv(params[r], K[f0 * L:f1 * L], V[f0 * L:f1 * L], Kc, Vc, None, km, vm, ws, ws.numel())
-        locals_.append((Kc, Vc, km, vm))
-    torch.cuda.synchronize()
-    Kc = sharded.assemble_compact([x[0] for x in locals_], kept)
-    Vc = sharded.assemble_compact([x[1] for x in locals_], kept)
+        P.avggt_build_kv_shard(params[r], K[f0 * L:f1 * L], V[f0 * L:f1 * L], gathered[r], slot_rows, None, sums, ws, ws.numel())
+        total += sums
     n_dropped = sum(dropped)
-    tot = max(n_dropped, 1)
-    kmean = sum(x[2].double() * n for x, n in zip(locals_, dropped)).div(tot).float()
-    vmean = sum(x[3].double() * n for x, n in zip(locals_, dropped)).div(tot).float()
+    Kc = torch.full((H, sum(kept), d), float("nan"), dtype=torch.bfloat16, device="cuda")
+    Vc = torch.full_like(Kc, float("nan"))
+    kmean = torch.zeros((H, d), device="cuda"); vmean = torch.zeros_like(kmean)
+    P.avggt_shard_assemble(params[0], gathered, kept, slot_rows, total, n_dropped, Kc, Vc, kmean, vmean)
+    torch.cuda.synchronize()
     O = torch.full_like(Q, float("nan"))
     for r, (f0, f1) in enumerate(ranges):
         _, aws = P.avggt_workspace_bytes(params[r])
@@ -51,21 +54,23 @@ def _shard_run(wl, world, keep_first=False, seed=0):
                                   ws, ws.numel())
         torch.cuda.synchronize()
         P.avggt_check_status(ws)
-    return Q, K, V, O, Kc, Vc
+    return Q, K, V, O, Kc, Vc, kmean, vmean
 
 
 @pytest.mark.parametrize("world", (2, 3))
 @pytest.mark.parametrize("keep_first", (False, True))
 def test_shards_reproduce_the_whole_sequence(world, keep_first):
     wl = inputs.Workload("shard", 5, 11, 13, 5, 4, 64, 4, 1, 2, "proj", keep_first_frame=int(keep_first))
-    Q, K, V, O, Kc, Vc = _shard_run(wl, world, keep_first, seed=8)
+    Q, K, V, O, Kc, Vc, kmean, vmean = _shard_run(wl, world, keep_first, seed=8)
     ocfg = orc.SGAConfig(wl.n_frames, wl.grid_h, wl.grid_w, wl.n_special, wl.n_heads, wl.head_dim, wl.sigma,
                          keep_first_frame=keep_first)
     Qh, Kh, Vh = (t.float().cpu().numpy() for t in (Q, K, V))
     # the assembled compact arrays are those of the unsharded layer, bit for bit
-    Kc_w, Vc_w, idx, _, _ = orc.build_kv(ocfg, Kh, Vh)
+    Kc_w, Vc_w, idx, kmean_w, vmean_w = orc.build_kv(ocfg, Kh, Vh)
     np.testing.assert_array_equal(Kc.float().cpu().numpy().transpose(1, 0, 2), Kc_w)
     np.testing.assert_array_equal(Vc.float().cpu().numpy().transpose(1, 0, 2), Vc_w)
+    for got_m, want_m, src in ((kmean, kmean_w, Kh), (vmean, vmean_w, Vh)):
+        assert np.abs(got_m.cpu().numpy().astype(np.float64) - want_m).max() <= 1e-5 * float(np.abs(src).mean())
     want = orc.global_attn_blocked(ocfg, Qh, Kh, Vh, np.arange(wl.n_tokens))
     got = O.float().cpu().numpy().astype(np.float64)
     assert np.isfinite(got).all()

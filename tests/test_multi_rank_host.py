@@ -1,8 +1,9 @@
-"""Host-side logic of the multi-GPU benchmark path, run as two gloo ranks on the CPU.
+"""Host-side logic of the multi-GPU path, run as two gloo ranks on the CPU.
 
-The path does not shard: `bench.py --gpus N` runs N independent replicas and reports the
-whole-job rate against the slowest rank's device time.  What needs no GPU is covered here:
-the max-over-ranks reduction, the aggregate, and that only rank 0 of the reference arm prints.
+`bench.py --gpus N` splits the frames of one problem over the ranks and reports the whole-job rate
+against the slowest rank's device time.  What needs no GPU is covered here: the max-over-ranks
+reduction, the aggregate, that only rank 0 of the reference arm prints, the frame split, and the
+two collectives of the exchange step on the exchange buffer's geometry.
 """
 
 import json
@@ -50,8 +51,8 @@ def test_max_over_ranks_two_gloo_ranks(tmp_path):
 def test_single_rank_needs_no_process_group():
     import bench
     assert bench.max_over_ranks([3.5, 2.0], "cpu", 1) == [3.5, 2.0]
-    # 2 replicas of 1000 queries per step, slowest step 4 ms -> 500k queries/s for the whole job
-    assert bench.whole_job_throughput(1000, 2, 4.0) == pytest.approx(5.0e5)
+    # 2000 queries over all ranks per step, slowest step 4 ms -> 500k queries/s for the whole job
+    assert bench.whole_job_throughput(2000, 4.0) == pytest.approx(5.0e5)
 
 
 def test_reference_arm_prints_on_rank_zero_only():
@@ -88,16 +89,18 @@ def test_shard_frames_covers_all_frames_evenly():
 def _exchange_main(rank, world, port, out_dir):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
     dist.init_process_group("gloo", rank=rank, world_size=world)
-    from paper_2512_02541_b200.sharded import combine_means, gather_compact
+    from paper_2512_02541_b200.sharded import exchange
     H, d = 3, 8
-    kept = [5, 9]                                  # uneven shards: padding on rank 0
-    dropped = [40, 24]
+    kept = [5, 9]                                  # uneven shards: padding rows in rank 0's slot
+    slot_rows = max(kept)
     gen = torch.Generator().manual_seed(100 + rank)
-    local = torch.randn((H, kept[rank], d), generator=gen).bfloat16()
-    mean = torch.randn((H, d), generator=gen)
-    full = gather_compact(local, kept)
-    m, total = combine_means(mean, dropped[rank])
-    torch.save({"local": local, "mean": mean, "full": full, "m": m, "total": total}, os.path.join(out_dir, f"x{rank}.pt"))
+    mine = torch.randn((2, H, kept[rank], d), generator=gen).bfloat16()
+    gathered = torch.zeros((world, 2, H, slot_rows, d), dtype=torch.bfloat16)
+    gathered[rank, :, :, :kept[rank]] = mine        # what the shard compaction writes: its own slot only
+    sums = torch.randn((2, H, d), generator=gen)
+    mine_sums = sums.clone()
+    exchange(gathered, rank, sums)
+    torch.save({"mine": mine, "mine_sums": mine_sums, "gathered": gathered, "sums": sums}, os.path.join(out_dir, f"x{rank}.pt"))
     dist.barrier()
     dist.destroy_process_group()
 
@@ -106,9 +109,11 @@ def test_exchange_step_two_gloo_ranks(tmp_path):
     world = 2
     mp.spawn(_exchange_main, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
     got = [torch.load(tmp_path / f"x{r}.pt") for r in range(world)]
-    want_full = torch.cat([got[0]["local"], got[1]["local"]], dim=1)          # rank order = ascending token order
-    want_mean = (got[0]["mean"].double() * 40 + got[1]["mean"].double() * 24) / 64
+    kept = [5, 9]
+    want_sums = got[0]["mine_sums"] + got[1]["mine_sums"]
     for r in range(world):
-        assert torch.equal(got[r]["full"], want_full)
-        assert got[r]["total"] == 64
-        assert torch.allclose(got[r]["m"].double(), want_mean, rtol=0, atol=1e-6)
+        g = got[r]["gathered"]
+        for o in range(world):                      # every rank holds every owner's slot, padding untouched
+            assert torch.equal(g[o, :, :, :kept[o]], got[o]["mine"])
+            assert not g[o, :, :, kept[o]:].any()
+        assert torch.allclose(got[r]["sums"], want_sums, rtol=0, atol=1e-6)

@@ -10,10 +10,12 @@ This file is collected last on purpose (a run that stops at the first failure ha
 every other test) and must pass alone in a fresh process as well as after the other tests.
 """
 
+import numpy as np
 import pytest
 import torch
 
 import paper_2512_02541_b200 as P
+from oracle import avggt_oracle as orc
 from paper_2512_02541_b200 import inputs
 
 pytestmark = pytest.mark.gpu
@@ -41,8 +43,14 @@ def test_noalloc_matches_build_kv_twice_in_a_row(wl):
             V = V - 3
         layer.build_kv(K, V)                       # the existing entry point, with a caller workspace
         Kc, Vc, idx, kmean, vmean = _buffers(layer)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         P.avggt_build_kv_noalloc(params, K, V, Kc, Vc, idx, kmean, vmean, stream)
         torch.cuda.synchronize()
+        # the call takes no device memory (checked from the second call on: the first one on a device may make
+        # the CUDA runtime load the kernels' code)
+        if call == 1:
+            assert torch.cuda.mem_get_info()[0] == free_before
         assert torch.equal(idx, layer.idx)
         assert torch.equal(Kc.view(torch.int16), layer.Kc.view(torch.int16))      # bit copies
         assert torch.equal(Vc.view(torch.int16), layer.Vc.view(torch.int16))
@@ -51,6 +59,16 @@ def test_noalloc_matches_build_kv_twice_in_a_row(wl):
             scale = max(float(src.float().abs().mean()), 1e-6)
             assert torch.isfinite(got).all()
             assert float((got - want).abs().max()) <= 1e-5 * scale
+        # and against the fp64 oracle directly
+        ocfg = orc.SGAConfig(wl.n_frames, wl.grid_h, wl.grid_w, wl.n_special, wl.n_heads, wl.head_dim, wl.sigma,
+                             diag=bool(wl.diag), mean_fill=wl.mean_fill)
+        Kh, Vh = K.float().cpu().numpy(), V.float().cpu().numpy()
+        Kc_w, Vc_w, idx_w, kmean_w, vmean_w = orc.build_kv(ocfg, Kh, Vh)
+        np.testing.assert_array_equal(idx.cpu().numpy(), idx_w)
+        np.testing.assert_array_equal(Kc.float().cpu().numpy().transpose(1, 0, 2).astype(np.float64), Kc_w)
+        np.testing.assert_array_equal(Vc.float().cpu().numpy().transpose(1, 0, 2).astype(np.float64), Vc_w)
+        for got, want, src in ((kmean, kmean_w, Kh), (vmean, vmean_w, Vh)):
+            assert np.abs(got.cpu().numpy().astype(np.float64) - want).max() <= 1e-5 * max(float(np.abs(src).mean()), 1e-6)
 
 
 def test_noalloc_rejects_problems_beyond_its_fixed_scratch():
