@@ -5,11 +5,9 @@
 //   warps 0-15  softmax.  Warpgroup g = 2 t + h works on query tile t and on
 //               columns [64 h, 64 h + 64) of every 128-key step; within it, warp q
 //               owns rows [32 q, 32 q + 32) (the tensor-memory lanes a warp may
-//               touch), one row per thread.  The two threads that share a row
-//               exchange their half-row maxima through shared memory every step
-//               and their partial sums once at the end.  Four softmax warps per
-//               scheduler keep the exponential unit busy while others wait on
-//               tensor memory, barriers or instruction fetch.
+//               touch), one row per thread.  Four softmax warps per scheduler keep
+//               the exponential unit busy while others wait on tensor memory or
+//               barriers.
 //   warp  16    TMA producer: Q tiles once, then the compacted K/V of the head
 //               through a ring of shared-memory stages (128-byte swizzle); the
 //               last two ring items are the K/V rows of the CTA's own queries
@@ -20,13 +18,23 @@
 //   warp  19    idle (it completes the fifth warpgroup so that registers can
 //               be moved to the softmax warpgroups)
 // Tensor memory per tile: S 128 columns (fp32), P 64 columns (bf16 pairs),
-// O 64 columns (fp32); 512 columns in all.  A softmax thread pulls its half row
-// of S into registers and frees S at once, so the next Q K^T runs under the
-// exponentials; P V of step j runs under the softmax of step j+1.  The
-// accumulator is rescaled lazily: only when the running maximum grew by more
-// than 2^8 since the last rescale.  The epilogue folds the diagonal and the
-// mean-fill column into the same normalisation:
+// O 64 columns (fp32); 512 columns in all.
+//
+// The softmax is software-pipelined over the key steps: while a thread turns
+// the scores of step j (held in registers) into probabilities, it pulls its
+// half row of S(j+1) out of tensor memory into the registers the exponentials
+// have just freed, and takes that half row's maximum at the end of the step.
+// Nothing but the partner's half-row maximum (written to shared memory one
+// whole step earlier) and the completion of P(j-1) V stands between two steps'
+// exponentials, so the four warps of a scheduler keep the exponential unit
+// fed without taking turns.  S(j+1) is released as soon as it is in registers:
+// Q K^T runs one step ahead, P V of step j under the exponentials of step j+1.
+// The accumulator is rescaled lazily: only when the running maximum grew by
+// more than 2^8 since the last rescale.  The epilogue folds the diagonal and
+// the mean-fill column into the same normalisation:
 //   O = (a_S O_S + p_d v_i + p_m vmean) / (a_S l_S + p_d + p_m).
+#include <mutex>
+
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -60,13 +68,6 @@ constexpr float kRescaleThreshold = 8.0f;   // log2 units
 #ifndef AVGGT_POLY_EIGHTHS
 #define AVGGT_POLY_EIGHTHS 0
 #endif
-// 1: the softmax warps of the two query tiles that share a scheduler take turns in the
-// exponential phase (two warps at a time saturate the unit), so that one tile's waits, loads,
-// maxima and stores run under the other tile's exponentials instead of all four warps
-// marching in step.
-#ifndef AVGGT_PINGPONG
-#define AVGGT_PINGPONG 1
-#endif
 constexpr int kPolyEighths = AVGGT_POLY_EIGHTHS;
 
 struct AttnArgs {
@@ -94,8 +95,8 @@ struct __align__(8) Barriers {
   uint64_t s_free[kQTiles];    // softmax -> MMA: S_t(j) has been read into registers
   uint64_t p_full[kQTiles];    // softmax -> MMA: P_t(j) stored (and O_t rescaled)
   uint64_t o_done[kQTiles];    // MMA -> softmax: P_t(j) V_j has completed
-  uint64_t turn[kQTiles][4];   // both warps of rows [32 q, 32 q + 32) of the other tile -> this tile's: the exponential unit is yours
   uint64_t pair[kQTiles][4];   // the two warps that share rows [32 q, 32 q + 32) of tile t: my half-row value is in shared memory
+  uint64_t mma_idle[kQTiles];  // MMA issuer t -> itself: every tcgen05.mma it issued has completed
   uint32_t tmem_base;
   uint32_t abort_flag;
 };
@@ -159,22 +160,6 @@ static_assert(kRegsSoftmax * kSoftmaxWarps + kRegsOther * (kThreads / 32 - kSoft
               "register budget after setmaxnreg exceeds the launch allocation");
 template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
-
-// Optional per-phase cycle counters of the softmax loop (a tuning aid; compiled out by default).
-#ifdef AVGGT_PHASE_TIMERS
-__device__ unsigned long long g_phase_cycles[4][4][8];   // [softmax warpgroup][warp][phase], CTA (0, 0)
-struct PhaseTimers {
-  unsigned long long acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  long long last = 0;
-  __device__ __forceinline__ void start() { last = clock64(); }
-  __device__ __forceinline__ void lap(int i) { const long long now = clock64(); acc[i] += now - last; last = now; }
-};
-#else
-struct PhaseTimers {
-  __device__ __forceinline__ void start() {}
-  __device__ __forceinline__ void lap(int) {}
-};
-#endif
 
 // What one CTA works on.
 struct CtaProblem {
@@ -293,12 +278,13 @@ __device__ __forceinline__ void issue_pv(const AttnArgs& a, Barriers* bars, uint
 }
 
 template <int t>
-__device__ __forceinline__ void mma_role(const AttnArgs& a, Barriers* bars, const SmemLayout& sm, uint32_t tmem) {
+__device__ __forceinline__ void mma_issue_loop(const AttnArgs& a, Barriers* bars, const SmemLayout& sm, uint32_t tmem) {
   static_assert(kStages >= 2, "the K ring must hold the tile in use and the next one");
   const int n_kv = a.n_kv_tiles;
   const uint64_t desc_q = umma_desc_sw128(smem_u32(sm.q[t]));
   const uint32_t k_base = smem_u32(sm.k), v_base = smem_u32(sm.v);
 
+  if (n_kv == 0) return;
   if (!wait_bar_warp(&bars->q_full, 0, bars, a, 20, 0)) return;
   if (!wait_bar_warp(&bars->k_full[0], 0, bars, a, 21, 0)) return;
   tc_fence_after();
@@ -320,6 +306,18 @@ __device__ __forceinline__ void mma_role(const AttnArgs& a, Barriers* bars, cons
     issue_pv<t>(a, bars, tmem, v_base, v_stage, j);
     if (++v_stage == kStages) { v_stage = 0; v_parity ^= 1; }
   }
+}
+
+// The issue loop, then (on every path out of it, a wait that ran out included) a wait until the
+// tensor core has finished everything this warp issued: the CTA must not free its tensor memory
+// or leave its shared memory while a tcgen05.mma still reads or writes them.
+template <int t>
+__device__ __forceinline__ void mma_role(const AttnArgs& a, Barriers* bars, const SmemLayout& sm, uint32_t tmem) {
+  mma_issue_loop<t>(a, bars, sm, tmem);
+  __syncwarp();
+  if (elect_one()) umma_commit(smem_u32(&bars->mma_idle[t]));
+  __syncwarp();
+  (void)wait_bar_warp(&bars->mma_idle[t], 0, bars, a, 70 + t, 0, false);
 }
 
 // ------------------------------------------------------------------ softmax warpgroup (128 threads per tile)
@@ -354,35 +352,29 @@ struct PairExchange {
   float final[kQTiles][2][2][kTileQ];   // [tile][which sum][half][row]: partial sums, once, in the epilogue
 };
 
-// 64 scores of one query row (a half row) -> bf16 probabilities, stored to tensor memory at tP,
-// relative to the reference maximum folded into neg_m2; adds to the sums for the normaliser (of
-// the rounded values) and for the log-sum-exp (unrounded).  Written pair by pair in dependency
-// order; the instruction scheduler interleaves the pairs.
+// 16 scores of one query row -> bf16 probabilities (8 packed pairs in pk), relative to the
+// reference maximum folded into neg_m2; adds to the sums for the normaliser (of the rounded
+// values) and for the log-sum-exp (unrounded).  Written pair by pair in dependency order; the
+// instruction scheduler interleaves the pairs.
 template <bool kLse, int kPoly>
-__device__ __forceinline__ void softmax_half_row(const uint32_t (&s)[64], uint64_t scale2, uint64_t neg_m2, uint64_t& sum2,
-                                                 uint64_t& sum_exact2, uint32_t tP) {
+__device__ __forceinline__ void exp_group(const uint32_t* s16, uint64_t scale2, uint64_t neg_m2, uint64_t& sum2,
+                                          uint64_t& sum_exact2, uint32_t* pk) {
 #pragma unroll
-  for (int g = 0; g < 4; ++g) {
-    uint32_t pk[8];   // P of 16 columns as bf16 pairs
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int c = 16 * g + 2 * i;
-      const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), scale2, neg_m2);
-      float p0, p1;
-      if (pair_uses_poly<kPoly>(i)) {
-        exp2_poly_pair(x2, p0, p1);
-      } else {
-        float x0, x1;
-        unpack_f32x2(x2, x0, x1);
-        p0 = ex2_approx(x0);
-        p1 = ex2_approx(x1);
-      }
-      const uint32_t w = pack_bf16x2(p0, p1);
-      pk[i] = w;
-      if (kLse) sum_exact2 = add_f32x2(sum_exact2, pack_f32x2(p0, p1));
-      sum2 = add_f32x2(sum2, pack_f32x2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)));
+  for (int i = 0; i < 8; ++i) {
+    const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s16[2 * i]), __uint_as_float(s16[2 * i + 1])), scale2, neg_m2);
+    float p0, p1;
+    if (pair_uses_poly<kPoly>(i)) {
+      exp2_poly_pair(x2, p0, p1);
+    } else {
+      float x0, x1;
+      unpack_f32x2(x2, x0, x1);
+      p0 = ex2_approx(x0);
+      p1 = ex2_approx(x1);
     }
-    tmem_st8(tP + g * 8, pk);
+    const uint32_t w = pack_bf16x2(p0, p1);
+    pk[i] = w;
+    if (kLse) sum_exact2 = add_f32x2(sum_exact2, pack_f32x2(p0, p1));
+    sum2 = add_f32x2(sum2, pack_f32x2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)));
   }
 }
 
@@ -396,46 +388,19 @@ struct SoftmaxThread {
   uint32_t tS, tP, tO;   // tensor-memory addresses of its half of S, P and O (lane included)
 };
 
-// Meeting point of the two warps that share the rows of `me`: returns once both have arrived for
-// the given phase (one phase per step, one more in the epilogue).  What either wrote to shared
-// memory before arriving is visible to the other afterwards.
-__device__ __forceinline__ bool pair_sync(uint32_t phase, const SoftmaxThread& me, Barriers* bars, const AttnArgs& a) {
+// The two warps that share the rows of `me` tell each other "my half-row value for this phase is
+// in shared memory" (one phase per step, one more in the epilogue).  What either wrote before
+// arriving is visible to the other once its wait returns.
+__device__ __forceinline__ void pair_arrive(const SoftmaxThread& me, Barriers* bars) {
   __syncwarp();
   if (me.lane == 0) mbar_arrive(smem_u32(&bars->pair[me.t][me.q]));
+}
+__device__ __forceinline__ bool pair_wait(uint32_t phase, const SoftmaxThread& me, Barriers* bars, const AttnArgs& a) {
   return wait_bar(&bars->pair[me.t][me.q], phase & 1, bars, a, 60 + me.t, phase);
 }
 
-// One step of the online softmax of half a query row: S_t(j) in tensor memory -> P_t(j) in
-// tensor memory, running reference maximum and partial sums updated.
-//
-// The half row's 64 scores are pulled into registers at once and the thread's share of S_t is
-// released, so that the next Q K^T runs under this step's exponentials.  The row maximum (of both
-// halves, exchanged with the partner thread) decides whether the reference maximum moves (lazy
-// rescale); both threads of a row take the same decision from the same numbers.
-// kPoly: pairs per eight whose exponential is a polynomial.  kLse: also keep the sum of the
-// unrounded exponentials, for the log-sum-exp output.  kMasked: columns >= valid are excluded
-// (valid counts from this thread's first column and may be <= 0).
-template <bool kMasked, bool kLse, int kPoly>
-__device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int valid, float scale_log2, float& m_used,
-                                             float& l_run, float& l_exact, Barriers* bars, PairExchange* px,
-                                             const AttnArgs& a, PhaseTimers& pt) {
-  uint32_t s[64];
-  {
-    uint32_t (&s2)[2][32] = reinterpret_cast<uint32_t (&)[2][32]>(s);
-    tmem_ld32(me.tS, s2[0]);
-    tmem_ld32(me.tS + 32, s2[1]);
-  }
-  tmem_wait_ld();
-  tc_fence_before();
-  __syncwarp();
-  if (me.lane == 0) mbar_arrive(smem_u32(&bars->s_free[me.t]));
-  pt.lap(1);
-
-  if (kMasked) {
-#pragma unroll
-    for (int i = 0; i < 64; ++i)
-      if (i >= valid) s[i] = __float_as_uint(-INFINITY);
-  }
+// Maximum of a half row of 64 scores held in registers.
+__device__ __forceinline__ float half_row_max(const uint32_t (&s)[64]) {
   float mx[2];
 #pragma unroll
   for (int c = 0; c < 2; ++c) {
@@ -443,10 +408,40 @@ __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int
 #pragma unroll
     for (int i = 2; i < 32; i += 2) mx[c] = max3(mx[c], __uint_as_float(s[32 * c + i]), __uint_as_float(s[32 * c + i + 1]));
   }
-  const float half_max = fmaxf(mx[0], mx[1]);
+  return fmaxf(mx[0], mx[1]);
+}
+
+// Scores in hand (in s, with their half-row maximum in half_max) become known to the partner:
+// columns at or beyond `valid` (counted from this thread's first column) are excluded first.
+template <bool kMasked>
+__device__ __forceinline__ void publish_half_max(const SoftmaxThread& me, int step, int valid, uint32_t (&s)[64],
+                                                 float& half_max, Barriers* bars, PairExchange* px) {
+  if (kMasked) {
+#pragma unroll
+    for (int i = 0; i < 64; ++i)
+      if (i >= valid) s[i] = __float_as_uint(-INFINITY);
+  }
+  half_max = half_row_max(s);
   // two slots, by step parity: the partner may still be reading the previous step's value
-  px->step[me.t][j & 1][me.h][me.r] = half_max;
-  if (!pair_sync(static_cast<uint32_t>(j), me, bars, a)) return false;
+  px->step[me.t][step & 1][me.h][me.r] = half_max;
+  pair_arrive(me, bars);
+}
+
+// One step of the online softmax of half a query row.  On entry s holds the thread's 64 scores
+// of step j and half_max their maximum (already published to the partner).  The step turns them
+// into P_t(j) in tensor memory and, when there is a next step, leaves the scores of step j+1 in
+// s (read from tensor memory into the registers the exponentials have freed) with their maximum
+// published.  The row maximum (of both halves) decides whether the reference maximum moves (lazy
+// rescale); both threads of a row take the same decision from the same numbers.
+// kHasNext: S_t(j+1) exists.  kMaskNext: its columns >= valid_next (counted from this thread's
+// first column; may be <= 0) are excluded.  kLse: also keep the sum of the unrounded
+// exponentials.  kPoly: pairs per eight whose exponential is a polynomial.
+template <bool kHasNext, bool kMaskNext, bool kLse, int kPoly>
+__device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int valid_next, float scale_log2,
+                                             uint32_t (&s)[64], float& half_max, float& m_used, float& l_run,
+                                             float& l_exact, Barriers* bars, PairExchange* px, const AttnArgs& a) {
+  // the partner's half-row maximum of this step: written while the previous step's exponentials ran
+  if (!pair_wait(static_cast<uint32_t>(j), me, bars, a)) return false;
   const float other_max = *reinterpret_cast<const volatile float*>(&px->step[me.t][j & 1][me.h ^ 1][me.r]);
   const float tile_max = fmaxf(half_max, other_max) * scale_log2;
   // lazy rescale: keep the old reference maximum unless the new one is far above it
@@ -458,40 +453,52 @@ __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int
     l_run *= alpha;
     if (kLse) l_exact *= alpha;
   }
-  const bool rescale = (j > 0) && __any_sync(0xffffffffu, jump);
-  pt.lap(2);
-
-  // P_t(j-1) must have been consumed, and O_t be at rest, before either is written
-  if (j > 0) {
+  if ((j > 0) && __any_sync(0xffffffffu, jump)) {   // rare: O_t must be at rest before it is rescaled
     if (!wait_bar(&bars->o_done[me.t], (j - 1) & 1, bars, a, 30 + me.t, j)) return false;
     tc_fence_after();
-  }
-  if (rescale) {   // this thread's 32 of the row's 64 accumulator columns
-    uint32_t o[32];
+    uint32_t o[32];   // this thread's 32 of the row's 64 accumulator columns
     tmem_ld32(me.tO, o);
     tmem_wait_ld();
 #pragma unroll
     for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
     tmem_st32(me.tO, o);
   }
-  pt.lap(3);
-#if AVGGT_PINGPONG
-  // this tile's turn on the exponential unit: the other tile's two warps on this scheduler have left their phase
-  if (!wait_bar(&bars->turn[me.t][me.q], j & 1, bars, a, 62 + me.t, j)) return false;
-#endif
-  pt.lap(6);
 
   // exponentials, rounded to bf16 for the value product; the normaliser sums the
   // rounded values so that numerator and denominator carry the same weights
   const uint64_t scale2 = pack_f32x2(scale_log2, scale_log2);
   const uint64_t neg_m2 = pack_f32x2(-m_used, -m_used);
   uint64_t sum2 = pack_f32x2(0.f, 0.f), sum_exact2 = pack_f32x2(0.f, 0.f);
-  softmax_half_row<kLse, kPoly>(s, scale2, neg_m2, sum2, sum_exact2, me.tP);
-#if AVGGT_PINGPONG
-  __syncwarp();
-  if (me.lane == 0) mbar_arrive(smem_u32(&bars->turn[me.t ^ 1][me.q]));
-#endif
-  pt.lap(4);
+  uint32_t (&s2)[2][32] = reinterpret_cast<uint32_t (&)[2][32]>(s);
+  {
+    uint32_t pk[16];
+    exp_group<kLse, kPoly>(&s[0], scale2, neg_m2, sum2, sum_exact2, &pk[0]);
+    exp_group<kLse, kPoly>(&s[16], scale2, neg_m2, sum2, sum_exact2, &pk[8]);
+    // P_t(j-1) must have been consumed before P_t(j) overwrites it
+    if (j > 0) {
+      if (!wait_bar(&bars->o_done[me.t], (j - 1) & 1, bars, a, 32 + me.t, j)) return false;
+      tc_fence_after();
+    }
+    tmem_st16(me.tP, pk);
+  }
+  if (kHasNext) {   // columns 0-31 of the next step into the registers just freed
+    if (!wait_bar(&bars->s_full[me.t], (j + 1) & 1, bars, a, 40 + me.t, j + 1)) return false;
+    tc_fence_after();
+    tmem_ld32(me.tS, s2[0]);
+  }
+#pragma unroll
+  for (int g = 2; g < 4; ++g) {   // stored in two pieces: with the next step's scores arriving, registers are scarce here
+    uint32_t pk[8];
+    exp_group<kLse, kPoly>(&s[16 * g], scale2, neg_m2, sum2, sum_exact2, pk);
+    tmem_st8(me.tP + 8 * g, pk);
+  }
+  if (kHasNext) {
+    tmem_ld32(me.tS + 32, s2[1]);
+    tmem_wait_ld64(s);
+    tc_fence_before();
+    __syncwarp();
+    if (me.lane == 0) mbar_arrive(smem_u32(&bars->s_free[me.t]));   // S_t(j+1) is in registers: Q K^T of step j+2 may go
+  }
 
   float sum_a, sum_b;
   unpack_f32x2(sum2, sum_a, sum_b);
@@ -504,7 +511,7 @@ __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int
   tc_fence_before();
   __syncwarp();
   if (me.lane == 0) mbar_arrive(smem_u32(&bars->p_full[me.t]));
-  pt.lap(5);
+  if (kHasNext) publish_half_max<kMaskNext>(me, j + 1, valid_next, s, half_max, bars, px);
   return true;
 }
 
@@ -527,31 +534,49 @@ __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, 
   float l_run = 0.f;          // this half's sum of the bf16-rounded 2^(scale_log2 * s - m_used): normaliser of O
   float l_exact = 0.f;        // the same sum without the rounding: log-sum-exp output only
   const bool want_lse = a.lse != nullptr;
-  PhaseTimers pt;
-  pt.start();
-#if AVGGT_PINGPONG
-  // tile 0 goes first: tile 1 hands it the first turn
-  if (t == 1 && lane == 0) mbar_arrive(smem_u32(&bars->turn[0][me.q]));
-#endif
+  // columns of the last step that exist, counted from this thread's first column (<= 0: none of its half)
+  const int valid_last = static_cast<int>(a.n_keys - static_cast<int64_t>(n_kv - 1) * kTileKV) - 64 * me.h;
+  const bool ragged = a.n_keys < static_cast<int64_t>(n_kv) * kTileKV;
 
-#pragma unroll 1
-  for (int j = 0; j < n_kv; ++j) {
-    if (!wait_bar(&bars->s_full[t], j & 1, bars, a, 40 + t, j)) return;
+  if (n_kv > 0) {
+    uint32_t s[64];
+    float half_max;
+    // scores of step 0
+    if (!wait_bar(&bars->s_full[t], 0, bars, a, 40 + t, 0)) return;
     tc_fence_after();
-    pt.lap(0);
-    const int valid_tile = static_cast<int>(a.n_keys - static_cast<int64_t>(j) * kTileKV);
-    const int valid = valid_tile - 64 * me.h;
-    bool ok;
-    // the masked (last, ragged) tile keeps every exponential on the special-function unit, where -inf gives an exact 0
-    if (valid_tile < kTileKV) ok = softmax_step<true, true, 0>(me, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a, pt);
-    else if (want_lse) ok = softmax_step<false, true, kPolyEighths>(me, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a, pt);
-    else ok = softmax_step<false, false, kPolyEighths>(me, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a, pt);
+    {
+      uint32_t (&s2)[2][32] = reinterpret_cast<uint32_t (&)[2][32]>(s);
+      tmem_ld32(me.tS, s2[0]);
+      tmem_ld32(me.tS + 32, s2[1]);
+    }
+    tmem_wait_ld64(s);
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&bars->s_free[t]));
+    if (n_kv == 1 && ragged) publish_half_max<true>(me, 0, valid_last, s, half_max, bars, px);
+    else publish_half_max<false>(me, 0, 0, s, half_max, bars, px);
+
+    // steps whose successor is a full tile, then the step before a ragged last tile, then the last step (which
+    // keeps every exponential on the special-function unit, where a masked score gives an exact 0)
+    const int n_plain = ragged ? n_kv - 2 : n_kv - 1;
+    int j = 0;
+    bool ok = true;
+    if (want_lse) {
+#pragma unroll 1
+      for (; j < n_plain && ok; ++j)
+        ok = softmax_step<true, false, true, kPolyEighths>(me, j, 0, a.scale_log2, s, half_max, m_used, l_run, l_exact, bars, px, a);
+    } else {
+#pragma unroll 1
+      for (; j < n_plain && ok; ++j)
+        ok = softmax_step<true, false, false, kPolyEighths>(me, j, 0, a.scale_log2, s, half_max, m_used, l_run, l_exact, bars, px, a);
+    }
     if (!ok) return;
+    if (j < n_kv - 1) {   // the successor is the ragged last tile
+      if (!softmax_step<true, true, true, kPolyEighths>(me, j, valid_last, a.scale_log2, s, half_max, m_used, l_run, l_exact, bars, px, a)) return;
+      ++j;
+    }
+    if (!softmax_step<false, false, true, 0>(me, j, 0, a.scale_log2, s, half_max, m_used, l_run, l_exact, bars, px, a)) return;
   }
-#ifdef AVGGT_PHASE_TIMERS
-  if (blockIdx.x == 0 && blockIdx.y == 0 && lane == 0)
-    for (int i = 0; i < 8; ++i) g_phase_cycles[warp >> 2][warp & 3][i] = pt.acc[i];
-#endif
 
   // ---- epilogue: diagonal and mean-fill terms, normalisation, store of this thread's 32 output dimensions
   const int head = cta.head;
@@ -565,14 +590,17 @@ __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, 
   // the row's sums: mine plus the partner's
   px->final[t][0][me.h][r] = l_run;
   px->final[t][1][me.h][r] = l_exact;
-  if (!pair_sync(static_cast<uint32_t>(n_kv), me, bars, a)) return;
+  pair_arrive(me, bars);
+  if (!pair_wait(static_cast<uint32_t>(n_kv), me, bars, a)) return;
   const float other_run = *reinterpret_cast<const volatile float*>(&px->final[t][0][me.h ^ 1][r]);
   const float other_exact = *reinterpret_cast<const volatile float*>(&px->final[t][1][me.h ^ 1][r]);
   l_run += other_run;
   l_exact += other_exact;
 
-  if (!wait_bar(&bars->o_done[t], (n_kv - 1) & 1, bars, a, 50 + t, n_kv)) return;
-  tc_fence_after();
+  if (n_kv > 0) {
+    if (!wait_bar(&bars->o_done[t], (n_kv - 1) & 1, bars, a, 50 + t, n_kv)) return;
+    tc_fence_after();
+  }
   if (!wait_bar(&bars->q_full, 0, bars, a, 52, 0)) return;   // completed long ago: makes the Q tile visible to this thread
   const int item = n_kv + t;                         // ring item holding this tile's own K/V rows
   const uint8_t* sKd = sm.k + (item % kStages) * kTileBytes;
@@ -621,8 +649,13 @@ __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, 
   const float w_s = a_s * inv_z, w_d = p_d * inv_z, w_m = p_m * inv_z;
 
   uint32_t o[32];
-  tmem_ld32(me.tO, o);
-  tmem_wait_ld();
+  if (n_kv > 0) {
+    tmem_ld32(me.tO, o);
+    tmem_wait_ld();
+  } else {   // no retained keys at all: the accumulator was never written
+#pragma unroll
+    for (int i = 0; i < 32; ++i) o[i] = 0u;
+  }
   if (row_valid) {
     uint4* dst = reinterpret_cast<uint4*>(a.O + (static_cast<size_t>(row) * pl.H + head) * kHeadDim) + 4 * me.h;
     const float4* vm = reinterpret_cast<const float4*>(a.vmean + head * kHeadDim) + 8 * me.h;
@@ -704,7 +737,7 @@ global_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       mbar_init(smem_u32(&bars.p_full[t]), kSoftmaxWarps / kQTiles);
       mbar_init(smem_u32(&bars.o_done[t]), 1);
       for (int w = 0; w < 4; ++w) mbar_init(smem_u32(&bars.pair[t][w]), 2);
-      for (int w = 0; w < 4; ++w) mbar_init(smem_u32(&bars.turn[t][w]), 2);
+      mbar_init(smem_u32(&bars.mma_idle[t]), 1);
     }
     bars.abort_flag = 0;
     fence_mbar_init();
@@ -728,6 +761,9 @@ global_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     else if (warp == kMmaWarp + 1) mma_role<1>(a, &bars, sm, tmem);
   }
 
+  // a role that left on a wait that ran out may have tensor-memory loads or stores in flight
+  tmem_wait_ld();
+  tmem_wait_st();
   tc_fence_before();
   __syncthreads();
   if (warp == kTmaWarp) tmem_dealloc(tmem, kTmemCols);
@@ -739,14 +775,31 @@ constexpr size_t kAttnSmemBytes = static_cast<size_t>(kTileBytes) * (kQTiles + 2
 
 size_t global_attn_ws_bytes(const Plan&, int) { return kAttnStatusBytes; }
 
-#ifdef AVGGT_PHASE_TIMERS
-// Tuning aid: copies the 4 x 4 x 8 phase counters of the last launch to the host.
-extern "C" int avggt_debug_phase_cycles(unsigned long long* out64) {
-  return cudaMemcpyFromSymbol(out64, g_phase_cycles, sizeof(g_phase_cycles)) == cudaSuccess ? 0 : -1;
-}
-#endif
-
 namespace {
+
+// Once per device: the dynamic shared-memory limit of the kernel, and a check that the launch allocates the
+// registers the role split hands out.  setmaxnreg.inc waits, without a time limit, for registers that other
+// warps release; if the compiler gave the kernel fewer than kRegsLaunch registers per thread the pool could
+// never cover the softmax warps' share and the kernel would hang, so such a build refuses to launch.
+cudaError_t prepare_kernel() {
+  static std::mutex mu;
+  static bool ready[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(mu);
+  if (ready[dev]) return cudaSuccess;
+  cudaFuncAttributes fa;
+  e = cudaFuncGetAttributes(&fa, global_attn_kernel);
+  if (e != cudaSuccess) return e;
+  if (fa.numRegs * (kThreads / 32) < kRegsSoftmax * kSoftmaxWarps + kRegsOther * (kThreads / 32 - kSoftmaxWarps))
+    return cudaErrorLaunchOutOfResources;
+  e = cudaFuncSetAttribute(global_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kAttnSmemBytes));
+  if (e != cudaSuccess) return e;
+  ready[dev] = true;
+  return cudaSuccess;
+}
 
 // Tensor maps and launch shared by the two entry points.  frame_mode: see AttnArgs.
 cudaError_t launch_attn(const Plan& pl, bool frame_mode, const void* Q, const void* K, const void* V, const void* Kc,
@@ -778,7 +831,7 @@ cudaError_t launch_attn(const Plan& pl, bool frame_mode, const void* Q, const vo
   bool good = make_tmap_bf16(&tm_q, Q, 2, tok_dims, tok_str, tok_box);
   good = good && make_tmap_bf16(&tm_k, reads_kv ? K : Q, 2, tok_dims, tok_str, tok_box);
   good = good && make_tmap_bf16(&tm_v, reads_kv ? V : Q, 2, tok_dims, tok_str, tok_box);
-  if (frame_mode) {
+  if (frame_mode || pl.M == 0) {
     tm_kc = tm_k;   // not read
     tm_vc = tm_v;
   } else {
@@ -790,9 +843,9 @@ cudaError_t launch_attn(const Plan& pl, bool frame_mode, const void* Q, const vo
   }
   if (!good) { *tmap_failed = true; return cudaSuccess; }
 
-  cudaError_t e = cudaMemsetAsync(ws, 0, kAttnStatusBytes, st);
+  cudaError_t e = prepare_kernel();
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(global_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kAttnSmemBytes));
+  e = cudaMemsetAsync(ws, 0, kAttnStatusBytes, st);
   if (e != cudaSuccess) return e;
   const int rows_per_cta = kQTiles * kTileQ;
   const int64_t rows = frame_mode ? pl.L : pl.n_tok;
