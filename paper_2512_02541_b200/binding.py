@@ -63,6 +63,37 @@ class AvggtError(RuntimeError):
 _LIB = None
 
 
+def load_library(path):
+    """ctypes handle of a build of the library at ``path`` with every entry point's signature declared."""
+    L = ctypes.CDLL(path)
+    vp, i64p, szp = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_size_t)
+    pp = ctypes.POINTER(AvggtParams)
+    sz, i64 = ctypes.c_size_t, ctypes.c_int64
+    signatures = {
+        "avggt_kv_count": [pp, i64p, i64p],
+        "avggt_workspace_bytes": [pp, szp, szp],
+        "avggt_build_kv": [pp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp],
+        "avggt_build_kv_noalloc": [pp, vp, vp, vp, vp, vp, vp, vp, vp],
+        "avggt_global_attn": [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp],
+        "avggt_frame_attn": [pp, vp, vp, vp, vp, vp, vp, sz, vp],
+        "avggt_build_kv_indexed": [pp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp],
+        "avggt_global_attn_indexed": [pp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp],
+        "avggt_global_attn_shard": [pp, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp],
+        "avggt_build_kv_shard": [pp, vp, vp, vp, i64, vp, vp, vp, sz, vp],
+        "avggt_shard_assemble": [pp, vp, ctypes.c_int32, i64p, i64, vp, i64, vp, vp, vp, vp, vp],
+        "avggt_check_status": [vp, ctypes.POINTER(ctypes.c_uint32)],
+        "avggt_strerror": [ctypes.c_int],
+        "avggt_last_cuda_error": [],
+        "avggt_version": [],
+    }
+    assert set(signatures) == set(EXPORTS)
+    for name, argtypes in signatures.items():
+        f = getattr(L, name)
+        f.argtypes = argtypes
+        f.restype = ctypes.c_char_p if name in ("avggt_strerror", "avggt_last_cuda_error", "avggt_version") else ctypes.c_int
+    return L
+
+
 def lib():
     """The loaded shared library (built in-tree on first use if stale or absent)."""
     global _LIB
@@ -75,34 +106,7 @@ def lib():
                 if not os.path.exists(_build.LIB):
                     raise
                 path = _build.LIB      # no compiler on this machine: use the library that shipped
-        L = ctypes.CDLL(path)
-        vp, i64p, szp = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_size_t)
-        pp = ctypes.POINTER(AvggtParams)
-        L.avggt_kv_count.argtypes = [pp, i64p, i64p]
-        L.avggt_workspace_bytes.argtypes = [pp, szp, szp]
-        L.avggt_build_kv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
-        L.avggt_build_kv_noalloc.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp]
-        L.avggt_build_kv_noalloc.restype = ctypes.c_int
-        L.avggt_global_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
-        L.avggt_frame_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
-        L.avggt_frame_attn.restype = ctypes.c_int
-        L.avggt_build_kv_indexed.argtypes = [pp, vp, ctypes.c_int64, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
-        L.avggt_build_kv_indexed.restype = ctypes.c_int
-        L.avggt_global_attn_indexed.argtypes = [pp, ctypes.c_int64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
-        L.avggt_global_attn_indexed.restype = ctypes.c_int
-        L.avggt_global_attn_shard.argtypes = [pp, ctypes.c_int64, ctypes.c_int64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
-        L.avggt_global_attn_shard.restype = ctypes.c_int
-        L.avggt_build_kv_shard.argtypes = [pp, vp, vp, vp, ctypes.c_int64, vp, vp, vp, ctypes.c_size_t, vp]
-        L.avggt_build_kv_shard.restype = ctypes.c_int
-        L.avggt_shard_assemble.argtypes = [pp, vp, ctypes.c_int32, i64p, ctypes.c_int64, vp, ctypes.c_int64, vp, vp, vp, vp, vp]
-        L.avggt_shard_assemble.restype = ctypes.c_int
-        L.avggt_check_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
-        L.avggt_strerror.argtypes = [ctypes.c_int]
-        for f in (L.avggt_kv_count, L.avggt_workspace_bytes, L.avggt_build_kv, L.avggt_global_attn, L.avggt_check_status):
-            f.restype = ctypes.c_int
-        for f in (L.avggt_strerror, L.avggt_last_cuda_error, L.avggt_version):
-            f.restype = ctypes.c_char_p
-        _LIB = L
+        _LIB = load_library(path)
     return _LIB
 
 

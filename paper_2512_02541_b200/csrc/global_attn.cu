@@ -5,9 +5,11 @@
 //   warps 0-15  softmax.  Warpgroup g = 2 t + h works on query tile t and on
 //               columns [64 h, 64 h + 64) of every 128-key step; within it, warp q
 //               owns rows [32 q, 32 q + 32) (the tensor-memory lanes a warp may
-//               touch), one row per thread.  Four softmax warps per scheduler keep
-//               the exponential unit busy while others wait on tensor memory or
-//               barriers.
+//               touch), one row per thread.  The two threads that share a row
+//               exchange their half-row maxima through shared memory every step
+//               and their partial sums once at the end.  Four softmax warps per
+//               scheduler keep the exponential unit busy while others wait on
+//               tensor memory, barriers or instruction fetch.
 //   warp  16    TMA producer: Q tiles once, then the compacted K/V of the head
 //               through a ring of shared-memory stages (128-byte swizzle); the
 //               last two ring items are the K/V rows of the CTA's own queries
@@ -18,20 +20,12 @@
 //   warp  19    idle (it completes the fifth warpgroup so that registers can
 //               be moved to the softmax warpgroups)
 // Tensor memory per tile: S 128 columns (fp32), P 64 columns (bf16 pairs),
-// O 64 columns (fp32); 512 columns in all.
-//
-// The softmax is software-pipelined over the key steps: while a thread turns
-// the scores of step j (held in registers) into probabilities, it pulls its
-// half row of S(j+1) out of tensor memory into the registers the exponentials
-// have just freed, and takes that half row's maximum at the end of the step.
-// Nothing but the partner's half-row maximum (written to shared memory one
-// whole step earlier) and the completion of P(j-1) V stands between two steps'
-// exponentials, so the four warps of a scheduler keep the exponential unit
-// fed without taking turns.  S(j+1) is released as soon as it is in registers:
-// Q K^T runs one step ahead, P V of step j under the exponentials of step j+1.
-// The accumulator is rescaled lazily: only when the running maximum grew by
-// more than 2^8 since the last rescale.  The epilogue folds the diagonal and
-// the mean-fill column into the same normalisation:
+// O 64 columns (fp32); 512 columns in all.  A softmax thread pulls its half row
+// of S into registers and frees S at once, so the next Q K^T runs under the
+// exponentials; P V of step j runs under the softmax of step j+1.  The
+// accumulator is rescaled lazily: only when the running maximum grew by more
+// than 2^8 since the last rescale.  The epilogue folds the diagonal and the
+// mean-fill column into the same normalisation:
 //   O = (a_S O_S + p_d v_i + p_m vmean) / (a_S l_S + p_d + p_m).
 #include <mutex>
 
@@ -68,6 +62,13 @@ constexpr float kRescaleThreshold = 8.0f;   // log2 units
 #ifndef AVGGT_POLY_EIGHTHS
 #define AVGGT_POLY_EIGHTHS 0
 #endif
+// 1: the softmax warps of the two query tiles that share a scheduler take turns in the
+// exponential phase (two warps at a time saturate the unit), so that one tile's waits, loads,
+// maxima and stores run under the other tile's exponentials instead of all four warps
+// marching in step.
+#ifndef AVGGT_PINGPONG
+#define AVGGT_PINGPONG 1
+#endif
 constexpr int kPolyEighths = AVGGT_POLY_EIGHTHS;
 
 struct AttnArgs {
@@ -95,6 +96,7 @@ struct __align__(8) Barriers {
   uint64_t s_free[kQTiles];    // softmax -> MMA: S_t(j) has been read into registers
   uint64_t p_full[kQTiles];    // softmax -> MMA: P_t(j) stored (and O_t rescaled)
   uint64_t o_done[kQTiles];    // MMA -> softmax: P_t(j) V_j has completed
+  uint64_t turn[kQTiles][4];   // both warps of rows [32 q, 32 q + 32) of the other tile -> this tile's: the exponential unit is yours
   uint64_t pair[kQTiles][4];   // the two warps that share rows [32 q, 32 q + 32) of tile t: my half-row value is in shared memory
   uint64_t mma_idle[kQTiles];  // MMA issuer t -> itself: every tcgen05.mma it issued has completed
   uint32_t tmem_base;
@@ -204,13 +206,21 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tm_q, const CUt
   }
   __syncwarp();
   int it = 0;
+  int k_issued = 0, v_issued = 0;   // ring items whose K / V copy has been issued
   int stage = 0;
   uint32_t empty_parity = 1;   // a fresh barrier passes the wait on the "previous" phase at once
   bool ok = true;
   for (; it < n_items; ++it) {
     ok = wait_bar_warp(&bars->k_empty[stage], empty_parity, bars, a, 10, it);
     if (!ok) break;
-    if (elect_one()) {
+#ifdef AVGGT_TEST_SKIP_K_LOAD
+    // Build for the wait-limit test only (never part of libavggt.so): the first thread block leaves out one K
+    // tile, so that the waits on it run out, the block reports the time-out and every role leaves in order.
+    const bool skip_load = it == AVGGT_TEST_SKIP_K_LOAD && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0;
+#else
+    constexpr bool skip_load = false;
+#endif
+    if (elect_one() && !skip_load) {
       const uint32_t kb = smem_u32(&bars->k_full[stage]);
       mbar_arrive_expect_tx(kb, kTileBytes);
       if (a.frame_mode) tma_load_2d(smem_u32(sm.k + stage * kTileBytes), tm_k, head * kHeadDim, cta.key_row0 + it * kTileKV, kb);
@@ -218,6 +228,7 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tm_q, const CUt
       else tma_load_2d(smem_u32(sm.k + stage * kTileBytes), tm_k, head * kHeadDim, q0 + (it - n_kv) * kTileQ, kb);
     }
     __syncwarp();
+    k_issued = it + 1;
     ok = wait_bar_warp(&bars->v_empty[stage], empty_parity, bars, a, 11, it);
     if (!ok) break;
     if (elect_one()) {
@@ -228,15 +239,17 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tm_q, const CUt
       else tma_load_2d(smem_u32(sm.v + stage * kTileBytes), tm_v, head * kHeadDim, q0 + (it - n_kv) * kTileQ, vb);
     }
     __syncwarp();
+    v_issued = it + 1;
     if (++stage == kStages) { stage = 0; empty_parity ^= 1; }
   }
   if (!ok) {
-    // let the copies still in flight land before the CTA gives up its shared memory
+    // let the copies still in flight land before the CTA gives up its shared memory: the last kStages
+    // issued into either ring (earlier ones completed before their stage was reused)
     (void)wait_bar_warp(&bars->q_full, 0, bars, a, 12, 0, false);
-    for (int back = 1; back <= kStages && it - back >= 0; ++back) {
-      const int jt = it - back;
-      (void)wait_bar_warp(&bars->k_full[jt % kStages], (jt / kStages) & 1, bars, a, 12, jt, false);
-      (void)wait_bar_warp(&bars->v_full[jt % kStages], (jt / kStages) & 1, bars, a, 12, jt, false);
+    for (int back = 1; back <= kStages; ++back) {
+      const int jk = k_issued - back, jv = v_issued - back;
+      if (jk >= 0) (void)wait_bar_warp(&bars->k_full[jk % kStages], (jk / kStages) & 1, bars, a, 12, jk, false);
+      if (jv >= 0) (void)wait_bar_warp(&bars->v_full[jv % kStages], (jv / kStages) & 1, bars, a, 13, jv, false);
     }
   }
 }
@@ -284,7 +297,7 @@ __device__ __forceinline__ void mma_issue_loop(const AttnArgs& a, Barriers* bars
   const uint64_t desc_q = umma_desc_sw128(smem_u32(sm.q[t]));
   const uint32_t k_base = smem_u32(sm.k), v_base = smem_u32(sm.v);
 
-  if (n_kv == 0) return;
+  if (n_kv == 0) return;   // no retained keys: the epilogue's two extra columns are the whole layer
   if (!wait_bar_warp(&bars->q_full, 0, bars, a, 20, 0)) return;
   if (!wait_bar_warp(&bars->k_full[0], 0, bars, a, 21, 0)) return;
   tc_fence_after();
@@ -352,29 +365,35 @@ struct PairExchange {
   float final[kQTiles][2][2][kTileQ];   // [tile][which sum][half][row]: partial sums, once, in the epilogue
 };
 
-// 16 scores of one query row -> bf16 probabilities (8 packed pairs in pk), relative to the
-// reference maximum folded into neg_m2; adds to the sums for the normaliser (of the rounded
-// values) and for the log-sum-exp (unrounded).  Written pair by pair in dependency order; the
-// instruction scheduler interleaves the pairs.
+// 64 scores of one query row (a half row) -> bf16 probabilities, stored to tensor memory at tP,
+// relative to the reference maximum folded into neg_m2; adds to the sums for the normaliser (of
+// the rounded values) and for the log-sum-exp (unrounded).  Written pair by pair in dependency
+// order; the instruction scheduler interleaves the pairs.
 template <bool kLse, int kPoly>
-__device__ __forceinline__ void exp_group(const uint32_t* s16, uint64_t scale2, uint64_t neg_m2, uint64_t& sum2,
-                                          uint64_t& sum_exact2, uint32_t* pk) {
+__device__ __forceinline__ void softmax_half_row(const uint32_t (&s)[64], uint64_t scale2, uint64_t neg_m2, uint64_t& sum2,
+                                                 uint64_t& sum_exact2, uint32_t tP) {
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s16[2 * i]), __uint_as_float(s16[2 * i + 1])), scale2, neg_m2);
-    float p0, p1;
-    if (pair_uses_poly<kPoly>(i)) {
-      exp2_poly_pair(x2, p0, p1);
-    } else {
-      float x0, x1;
-      unpack_f32x2(x2, x0, x1);
-      p0 = ex2_approx(x0);
-      p1 = ex2_approx(x1);
+  for (int g = 0; g < 4; ++g) {
+    uint32_t pk[8];   // P of 16 columns as bf16 pairs
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int c = 16 * g + 2 * i;
+      const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), scale2, neg_m2);
+      float p0, p1;
+      if (pair_uses_poly<kPoly>(i)) {
+        exp2_poly_pair(x2, p0, p1);
+      } else {
+        float x0, x1;
+        unpack_f32x2(x2, x0, x1);
+        p0 = ex2_approx(x0);
+        p1 = ex2_approx(x1);
+      }
+      const uint32_t w = pack_bf16x2(p0, p1);
+      pk[i] = w;
+      if (kLse) sum_exact2 = add_f32x2(sum_exact2, pack_f32x2(p0, p1));
+      sum2 = add_f32x2(sum2, pack_f32x2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)));
     }
-    const uint32_t w = pack_bf16x2(p0, p1);
-    pk[i] = w;
-    if (kLse) sum_exact2 = add_f32x2(sum_exact2, pack_f32x2(p0, p1));
-    sum2 = add_f32x2(sum2, pack_f32x2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)));
+    tmem_st8(tP + g * 8, pk);
   }
 }
 
@@ -388,19 +407,45 @@ struct SoftmaxThread {
   uint32_t tS, tP, tO;   // tensor-memory addresses of its half of S, P and O (lane included)
 };
 
-// The two warps that share the rows of `me` tell each other "my half-row value for this phase is
-// in shared memory" (one phase per step, one more in the epilogue).  What either wrote before
-// arriving is visible to the other once its wait returns.
-__device__ __forceinline__ void pair_arrive(const SoftmaxThread& me, Barriers* bars) {
+// Meeting point of the two warps that share the rows of `me`: returns once both have arrived for
+// the given phase (one phase per step, one more in the epilogue).  What either wrote to shared
+// memory before arriving is visible to the other afterwards.
+__device__ __forceinline__ bool pair_sync(uint32_t phase, const SoftmaxThread& me, Barriers* bars, const AttnArgs& a) {
   __syncwarp();
   if (me.lane == 0) mbar_arrive(smem_u32(&bars->pair[me.t][me.q]));
-}
-__device__ __forceinline__ bool pair_wait(uint32_t phase, const SoftmaxThread& me, Barriers* bars, const AttnArgs& a) {
   return wait_bar(&bars->pair[me.t][me.q], phase & 1, bars, a, 60 + me.t, phase);
 }
 
-// Maximum of a half row of 64 scores held in registers.
-__device__ __forceinline__ float half_row_max(const uint32_t (&s)[64]) {
+// One step of the online softmax of half a query row: S_t(j) in tensor memory -> P_t(j) in
+// tensor memory, running reference maximum and partial sums updated.
+//
+// The half row's 64 scores are pulled into registers at once and the thread's share of S_t is
+// released, so that the next Q K^T runs under this step's exponentials.  The row maximum (of both
+// halves, exchanged with the partner thread) decides whether the reference maximum moves (lazy
+// rescale); both threads of a row take the same decision from the same numbers.
+// kPoly: pairs per eight whose exponential is a polynomial.  kLse: also keep the sum of the
+// unrounded exponentials, for the log-sum-exp output.  kMasked: columns >= valid are excluded
+// (valid counts from this thread's first column and may be <= 0).
+template <bool kMasked, bool kLse, int kPoly>
+__device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int valid, float scale_log2, float& m_used,
+                                             float& l_run, float& l_exact, Barriers* bars, PairExchange* px,
+                                             const AttnArgs& a) {
+  uint32_t s[64];
+  {
+    uint32_t (&s2)[2][32] = reinterpret_cast<uint32_t (&)[2][32]>(s);
+    tmem_ld32(me.tS, s2[0]);
+    tmem_ld32(me.tS + 32, s2[1]);
+  }
+  tmem_wait_ld();
+  tc_fence_before();
+  __syncwarp();
+  if (me.lane == 0) mbar_arrive(smem_u32(&bars->s_free[me.t]));
+
+  if (kMasked) {
+#pragma unroll
+    for (int i = 0; i < 64; ++i)
+      if (i >= valid) s[i] = __float_as_uint(-INFINITY);
+  }
   float mx[2];
 #pragma unroll
   for (int c = 0; c < 2; ++c) {
@@ -408,40 +453,10 @@ __device__ __forceinline__ float half_row_max(const uint32_t (&s)[64]) {
 #pragma unroll
     for (int i = 2; i < 32; i += 2) mx[c] = max3(mx[c], __uint_as_float(s[32 * c + i]), __uint_as_float(s[32 * c + i + 1]));
   }
-  return fmaxf(mx[0], mx[1]);
-}
-
-// Scores in hand (in s, with their half-row maximum in half_max) become known to the partner:
-// columns at or beyond `valid` (counted from this thread's first column) are excluded first.
-template <bool kMasked>
-__device__ __forceinline__ void publish_half_max(const SoftmaxThread& me, int step, int valid, uint32_t (&s)[64],
-                                                 float& half_max, Barriers* bars, PairExchange* px) {
-  if (kMasked) {
-#pragma unroll
-    for (int i = 0; i < 64; ++i)
-      if (i >= valid) s[i] = __float_as_uint(-INFINITY);
-  }
-  half_max = half_row_max(s);
+  const float half_max = fmaxf(mx[0], mx[1]);
   // two slots, by step parity: the partner may still be reading the previous step's value
-  px->step[me.t][step & 1][me.h][me.r] = half_max;
-  pair_arrive(me, bars);
-}
-
-// One step of the online softmax of half a query row.  On entry s holds the thread's 64 scores
-// of step j and half_max their maximum (already published to the partner).  The step turns them
-// into P_t(j) in tensor memory and, when there is a next step, leaves the scores of step j+1 in
-// s (read from tensor memory into the registers the exponentials have freed) with their maximum
-// published.  The row maximum (of both halves) decides whether the reference maximum moves (lazy
-// rescale); both threads of a row take the same decision from the same numbers.
-// kHasNext: S_t(j+1) exists.  kMaskNext: its columns >= valid_next (counted from this thread's
-// first column; may be <= 0) are excluded.  kLse: also keep the sum of the unrounded
-// exponentials.  kPoly: pairs per eight whose exponential is a polynomial.
-template <bool kHasNext, bool kMaskNext, bool kLse, int kPoly>
-__device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int valid_next, float scale_log2,
-                                             uint32_t (&s)[64], float& half_max, float& m_used, float& l_run,
-                                             float& l_exact, Barriers* bars, PairExchange* px, const AttnArgs& a) {
-  // the partner's half-row maximum of this step: written while the previous step's exponentials ran
-  if (!pair_wait(static_cast<uint32_t>(j), me, bars, a)) return false;
+  px->step[me.t][j & 1][me.h][me.r] = half_max;
+  if (!pair_sync(static_cast<uint32_t>(j), me, bars, a)) return false;
   const float other_max = *reinterpret_cast<const volatile float*>(&px->step[me.t][j & 1][me.h ^ 1][me.r]);
   const float tile_max = fmaxf(half_max, other_max) * scale_log2;
   // lazy rescale: keep the old reference maximum unless the new one is far above it
@@ -453,52 +468,36 @@ __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int
     l_run *= alpha;
     if (kLse) l_exact *= alpha;
   }
-  if ((j > 0) && __any_sync(0xffffffffu, jump)) {   // rare: O_t must be at rest before it is rescaled
+  const bool rescale = (j > 0) && __any_sync(0xffffffffu, jump);
+
+  // P_t(j-1) must have been consumed, and O_t be at rest, before either is written
+  if (j > 0) {
     if (!wait_bar(&bars->o_done[me.t], (j - 1) & 1, bars, a, 30 + me.t, j)) return false;
     tc_fence_after();
-    uint32_t o[32];   // this thread's 32 of the row's 64 accumulator columns
+  }
+  if (rescale) {   // this thread's 32 of the row's 64 accumulator columns
+    uint32_t o[32];
     tmem_ld32(me.tO, o);
     tmem_wait_ld();
 #pragma unroll
     for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
     tmem_st32(me.tO, o);
   }
+#if AVGGT_PINGPONG
+  // this tile's turn on the exponential unit: the other tile's two warps on this scheduler have left their phase
+  if (!wait_bar(&bars->turn[me.t][me.q], j & 1, bars, a, 62 + me.t, j)) return false;
+#endif
 
   // exponentials, rounded to bf16 for the value product; the normaliser sums the
   // rounded values so that numerator and denominator carry the same weights
   const uint64_t scale2 = pack_f32x2(scale_log2, scale_log2);
   const uint64_t neg_m2 = pack_f32x2(-m_used, -m_used);
   uint64_t sum2 = pack_f32x2(0.f, 0.f), sum_exact2 = pack_f32x2(0.f, 0.f);
-  uint32_t (&s2)[2][32] = reinterpret_cast<uint32_t (&)[2][32]>(s);
-  {
-    uint32_t pk[16];
-    exp_group<kLse, kPoly>(&s[0], scale2, neg_m2, sum2, sum_exact2, &pk[0]);
-    exp_group<kLse, kPoly>(&s[16], scale2, neg_m2, sum2, sum_exact2, &pk[8]);
-    // P_t(j-1) must have been consumed before P_t(j) overwrites it
-    if (j > 0) {
-      if (!wait_bar(&bars->o_done[me.t], (j - 1) & 1, bars, a, 32 + me.t, j)) return false;
-      tc_fence_after();
-    }
-    tmem_st16(me.tP, pk);
-  }
-  if (kHasNext) {   // columns 0-31 of the next step into the registers just freed
-    if (!wait_bar(&bars->s_full[me.t], (j + 1) & 1, bars, a, 40 + me.t, j + 1)) return false;
-    tc_fence_after();
-    tmem_ld32(me.tS, s2[0]);
-  }
-#pragma unroll
-  for (int g = 2; g < 4; ++g) {   // stored in two pieces: with the next step's scores arriving, registers are scarce here
-    uint32_t pk[8];
-    exp_group<kLse, kPoly>(&s[16 * g], scale2, neg_m2, sum2, sum_exact2, pk);
-    tmem_st8(me.tP + 8 * g, pk);
-  }
-  if (kHasNext) {
-    tmem_ld32(me.tS + 32, s2[1]);
-    tmem_wait_ld64(s);
-    tc_fence_before();
-    __syncwarp();
-    if (me.lane == 0) mbar_arrive(smem_u32(&bars->s_free[me.t]));   // S_t(j+1) is in registers: Q K^T of step j+2 may go
-  }
+  softmax_half_row<kLse, kPoly>(s, scale2, neg_m2, sum2, sum_exact2, me.tP);
+#if AVGGT_PINGPONG
+  __syncwarp();
+  if (me.lane == 0) mbar_arrive(smem_u32(&bars->turn[me.t ^ 1][me.q]));
+#endif
 
   float sum_a, sum_b;
   unpack_f32x2(sum2, sum_a, sum_b);
@@ -511,7 +510,6 @@ __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int
   tc_fence_before();
   __syncwarp();
   if (me.lane == 0) mbar_arrive(smem_u32(&bars->p_full[me.t]));
-  if (kHasNext) publish_half_max<kMaskNext>(me, j + 1, valid_next, s, half_max, bars, px);
   return true;
 }
 
@@ -534,48 +532,23 @@ __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, 
   float l_run = 0.f;          // this half's sum of the bf16-rounded 2^(scale_log2 * s - m_used): normaliser of O
   float l_exact = 0.f;        // the same sum without the rounding: log-sum-exp output only
   const bool want_lse = a.lse != nullptr;
-  // columns of the last step that exist, counted from this thread's first column (<= 0: none of its half)
-  const int valid_last = static_cast<int>(a.n_keys - static_cast<int64_t>(n_kv - 1) * kTileKV) - 64 * me.h;
-  const bool ragged = a.n_keys < static_cast<int64_t>(n_kv) * kTileKV;
+#if AVGGT_PINGPONG
+  // tile 0 goes first: tile 1 hands it the first turn
+  if (t == 1 && lane == 0) mbar_arrive(smem_u32(&bars->turn[0][me.q]));
+#endif
 
-  if (n_kv > 0) {
-    uint32_t s[64];
-    float half_max;
-    // scores of step 0
-    if (!wait_bar(&bars->s_full[t], 0, bars, a, 40 + t, 0)) return;
+#pragma unroll 1
+  for (int j = 0; j < n_kv; ++j) {
+    if (!wait_bar(&bars->s_full[t], j & 1, bars, a, 40 + t, j)) return;
     tc_fence_after();
-    {
-      uint32_t (&s2)[2][32] = reinterpret_cast<uint32_t (&)[2][32]>(s);
-      tmem_ld32(me.tS, s2[0]);
-      tmem_ld32(me.tS + 32, s2[1]);
-    }
-    tmem_wait_ld64(s);
-    tc_fence_before();
-    __syncwarp();
-    if (lane == 0) mbar_arrive(smem_u32(&bars->s_free[t]));
-    if (n_kv == 1 && ragged) publish_half_max<true>(me, 0, valid_last, s, half_max, bars, px);
-    else publish_half_max<false>(me, 0, 0, s, half_max, bars, px);
-
-    // steps whose successor is a full tile, then the step before a ragged last tile, then the last step (which
-    // keeps every exponential on the special-function unit, where a masked score gives an exact 0)
-    const int n_plain = ragged ? n_kv - 2 : n_kv - 1;
-    int j = 0;
-    bool ok = true;
-    if (want_lse) {
-#pragma unroll 1
-      for (; j < n_plain && ok; ++j)
-        ok = softmax_step<true, false, true, kPolyEighths>(me, j, 0, a.scale_log2, s, half_max, m_used, l_run, l_exact, bars, px, a);
-    } else {
-#pragma unroll 1
-      for (; j < n_plain && ok; ++j)
-        ok = softmax_step<true, false, false, kPolyEighths>(me, j, 0, a.scale_log2, s, half_max, m_used, l_run, l_exact, bars, px, a);
-    }
+    const int valid_tile = static_cast<int>(a.n_keys - static_cast<int64_t>(j) * kTileKV);
+    const int valid = valid_tile - 64 * me.h;
+    bool ok;
+    // the masked (last, ragged) tile keeps every exponential on the special-function unit, where -inf gives an exact 0
+    if (valid_tile < kTileKV) ok = softmax_step<true, true, 0>(me, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a);
+    else if (want_lse) ok = softmax_step<false, true, kPolyEighths>(me, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a);
+    else ok = softmax_step<false, false, kPolyEighths>(me, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a);
     if (!ok) return;
-    if (j < n_kv - 1) {   // the successor is the ragged last tile
-      if (!softmax_step<true, true, true, kPolyEighths>(me, j, valid_last, a.scale_log2, s, half_max, m_used, l_run, l_exact, bars, px, a)) return;
-      ++j;
-    }
-    if (!softmax_step<false, false, true, 0>(me, j, 0, a.scale_log2, s, half_max, m_used, l_run, l_exact, bars, px, a)) return;
   }
 
   // ---- epilogue: diagonal and mean-fill terms, normalisation, store of this thread's 32 output dimensions
@@ -590,8 +563,7 @@ __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, 
   // the row's sums: mine plus the partner's
   px->final[t][0][me.h][r] = l_run;
   px->final[t][1][me.h][r] = l_exact;
-  pair_arrive(me, bars);
-  if (!pair_wait(static_cast<uint32_t>(n_kv), me, bars, a)) return;
+  if (!pair_sync(static_cast<uint32_t>(n_kv), me, bars, a)) return;
   const float other_run = *reinterpret_cast<const volatile float*>(&px->final[t][0][me.h ^ 1][r]);
   const float other_exact = *reinterpret_cast<const volatile float*>(&px->final[t][1][me.h ^ 1][r]);
   l_run += other_run;
@@ -737,6 +709,7 @@ global_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       mbar_init(smem_u32(&bars.p_full[t]), kSoftmaxWarps / kQTiles);
       mbar_init(smem_u32(&bars.o_done[t]), 1);
       for (int w = 0; w < 4; ++w) mbar_init(smem_u32(&bars.pair[t][w]), 2);
+      for (int w = 0; w < 4; ++w) mbar_init(smem_u32(&bars.turn[t][w]), 2);
       mbar_init(smem_u32(&bars.mma_idle[t]), 1);
     }
     bars.abort_flag = 0;
