@@ -55,7 +55,10 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
     assert code == binding.AVGGT_ERR_DEVICE_TIMEOUT
     flag, block, site, iteration = detail
     assert flag == 1 and block == 0                       # the first thread block gave up ...
-    assert site in (24, 25) and iteration == 0            # ... in an MMA issuer's wait for K tile 1 (the one left out)
+    # ... in whichever of its roles had waited longest on the consequences of the missing K tile: the producer
+    # on a ring stage that is never released (sites 10, 11), an MMA issuer on the tile itself (24, 25) or a
+    # softmax warp on the scores of step 1 (40, 41); all within the first ring cycle
+    assert site in (10, 11, 24, 25, 40, 41) and iteration <= 3
     # the blocks of the last head start after the time-out and leave at once: their rows were never written
     assert torch.isnan(O[:, wl.n_heads - 1].float()).any()
 
