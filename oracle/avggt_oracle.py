@@ -328,6 +328,11 @@ def global_attn_indexed(cfg, idx, Q, K, V, rows=None, return_lse=False):
     retained set, the query's own column if it is in D (diag), one mean pair over D entering with
     weight 1 or with the count of columns it stands for (mean_fill 1 / 2), one shared softmax.
     The retained keys are taken in ascending token order.
+
+    An empty ``idx`` is the paper's G2M variant (Sec. 5.4, "Effect of the Early Global Attention
+    Layers"): every Key/Value, special tokens included, is replaced by the one mean pair over the
+    whole sequence.  With ``diag`` off every output row is then that mean Value; with ``diag`` on
+    each query sees its own column and the mean pair.
     """
     Q = np.asarray(Q, dtype=np.float64)
     K = np.asarray(K, dtype=np.float64)
@@ -335,7 +340,7 @@ def global_attn_indexed(cfg, idx, Q, K, V, rows=None, return_lse=False):
     H, d = cfg.n_heads, cfg.head_dim
     assert Q.shape == (cfg.n_tokens, H, d) and K.shape == Q.shape and V.shape == Q.shape
     idx = np.sort(np.asarray(idx, dtype=np.int64))
-    assert len(idx) > 0 and len(np.unique(idx)) == len(idx) and idx[0] >= 0 and idx[-1] < cfg.n_tokens
+    assert len(np.unique(idx)) == len(idx) and (len(idx) == 0 or (idx[0] >= 0 and idx[-1] < cfg.n_tokens))
     scale = cfg.scale
     dropped = np.ones(cfg.n_tokens, dtype=bool)
     dropped[idx] = False

@@ -370,8 +370,8 @@ struct PairExchange {
 // the rounded values) and for the log-sum-exp (unrounded).  Written pair by pair in dependency
 // order; the instruction scheduler interleaves the pairs.
 template <bool kLse, int kPoly>
-__device__ __forceinline__ void softmax_half_row(const uint32_t (&s)[64], uint64_t scale2, uint64_t neg_m2, uint64_t& sum2,
-                                                 uint64_t& sum_exact2, uint32_t tP) {
+__device__ __forceinline__ void softmax_half_row(const uint32_t (&s)[64], uint64_t scale2, uint64_t neg_m2, float& sum_lo,
+                                                 float& sum_hi, uint64_t& sum_exact2, uint32_t tP) {
 #pragma unroll
   for (int g = 0; g < 4; ++g) {
     uint32_t pk[8];   // P of 16 columns as bf16 pairs
@@ -391,7 +391,7 @@ __device__ __forceinline__ void softmax_half_row(const uint32_t (&s)[64], uint64
       const uint32_t w = pack_bf16x2(p0, p1);
       pk[i] = w;
       if (kLse) sum_exact2 = add_f32x2(sum_exact2, pack_f32x2(p0, p1));
-      sum2 = add_f32x2(sum2, pack_f32x2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)));
+      add_bf16x2_to_f32(w, sum_lo, sum_hi);
     }
     tmem_st8(tP + g * 8, pk);
   }
@@ -492,17 +492,17 @@ __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int
   // rounded values so that numerator and denominator carry the same weights
   const uint64_t scale2 = pack_f32x2(scale_log2, scale_log2);
   const uint64_t neg_m2 = pack_f32x2(-m_used, -m_used);
-  uint64_t sum2 = pack_f32x2(0.f, 0.f), sum_exact2 = pack_f32x2(0.f, 0.f);
-  softmax_half_row<kLse, kPoly>(s, scale2, neg_m2, sum2, sum_exact2, me.tP);
+  float sum_lo = 0.f, sum_hi = 0.f;   // even and odd columns
+  uint64_t sum_exact2 = pack_f32x2(0.f, 0.f);
+  softmax_half_row<kLse, kPoly>(s, scale2, neg_m2, sum_lo, sum_hi, sum_exact2, me.tP);
 #if AVGGT_PINGPONG
   __syncwarp();
   if (me.lane == 0) mbar_arrive(smem_u32(&bars->turn[me.t ^ 1][me.q]));
 #endif
 
-  float sum_a, sum_b;
-  unpack_f32x2(sum2, sum_a, sum_b);
-  l_run += sum_a + sum_b;
+  l_run += sum_lo + sum_hi;
   if (kLse) {
+    float sum_a, sum_b;
     unpack_f32x2(sum_exact2, sum_a, sum_b);
     l_exact += sum_a + sum_b;
   }

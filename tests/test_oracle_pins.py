@@ -410,3 +410,26 @@ def test_indexed_keeping_everything_is_dense_sdpa():
     ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv)[0].permute(1, 0, 2).numpy()
     np.testing.assert_allclose(orc.global_attn_indexed(cfg, np.arange(cfg.n_tokens), Q, K, V), ref, rtol=0, atol=1e-12)
 
+
+
+@pytest.mark.parametrize("mean_fill", (1, 2))
+def test_indexed_with_nothing_retained_is_the_mean_value(mean_fill):
+    """G2M (Sec. 5.4): all Keys/Values replaced by one mean pair.  Without the diagonal the softmax has a
+    single column, so every output row is the plain mean of V over all tokens, whatever Q and K are."""
+    cfg = _tiny(4, False, mean_fill)
+    Q, K, V = _rand_qkv(cfg, seed=61)
+    got, lse = orc.global_attn_indexed(cfg, np.zeros(0, dtype=np.int64), Q, K, V, return_lse=True)
+    want = np.broadcast_to(V.mean(axis=0), got.shape)
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-12)
+    # one column of logit scale * q.kmean (+ ln N in fill mode): the normaliser is that logit itself
+    lm = cfg.scale * np.einsum("nhd,hd->nh", Q, K.mean(axis=0)) + (math.log(cfg.n_tokens) if mean_fill == 2 else 0.0)
+    np.testing.assert_allclose(lse, lm, rtol=0, atol=1e-10)
+
+
+@pytest.mark.parametrize("mean_fill", (0, 1, 2))
+def test_indexed_with_nothing_retained_and_the_diagonal_matches_filled_matrix_brute_force(mean_fill):
+    cfg = _tiny(2, True, mean_fill)
+    Q, K, V = _rand_qkv(cfg, seed=63)
+    D = np.ones(cfg.n_tokens, dtype=bool)
+    np.testing.assert_allclose(orc.global_attn_indexed(cfg, np.zeros(0, dtype=np.int64), Q, K, V),
+                               _brute_force(cfg, Q, K, V, D=D), rtol=0, atol=1e-12)
