@@ -186,7 +186,9 @@ int avggt_global_attn(const avggt_params* p, const void* Q, const void* K, const
  * random, norm-ranked or feature-based picks).  `idx` lists the n_kept retained tokens; every
  * other token is in D, whatever its kind (list the special tokens to keep them).  Diagonal
  * preservation, the mean pair over D and the shared softmax are as in Sec. 4.3.  Of `p`, sigma
- * and flags play no part but must be valid.
+ * and flags play no part but must be valid.  n_kept = 0 is allowed when diag or mean_fill is on: it
+ * is the G2M variant of Sec. 5.4 ("Effect of the Early Global Attention Layers"), in which one mean
+ * pair over the whole sequence stands for every Key/Value (idx, Kc and Vc may then be NULL).
  *
  * avggt_build_kv_indexed
  *   idx            device, int32 [n_kept], strictly ascending token indices in [0, N*L).  The list

@@ -196,7 +196,9 @@ int avggt_global_attn(const avggt_params* p, const void* Q, const void* K, const
 static int make_indexed_plan(const avggt_params* p, int64_t n_kept, Plan* pl) {
   int rc = make_plan(p, pl);
   if (rc != AVGGT_OK) return rc;
-  if (n_kept < 1 || n_kept > pl->n_tok) return AVGGT_ERR_INVALID_ARG;
+  if (n_kept < 0 || n_kept > pl->n_tok) return AVGGT_ERR_INVALID_ARG;
+  // nothing retained (the G2M variant of Sec. 5.4): some column must remain for the softmax
+  if (n_kept == 0 && pl->diag == 0 && pl->mean_fill == 0) return AVGGT_ERR_INVALID_ARG;
   pl->M = n_kept;
   pl->n_dropped = pl->n_tok - n_kept;
   pl->keep_first = 0;

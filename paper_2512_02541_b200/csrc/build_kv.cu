@@ -237,10 +237,11 @@ cudaError_t launch_build_kv(const Plan& pl, int sm_count, const void* K, const v
                             int32_t* idx, float* kmean, float* vmean, void* ws, cudaStream_t st,
                             const int32_t* caller_idx, int32_t* slot_of_token, int64_t kc_rows, bool sums_only) {
   if (kc_rows <= 0) kc_rows = pl.M;
-  if (caller_idx != nullptr) {
+  if (slot_of_token != nullptr) {
     // caller-chosen retained set: build the token -> compact position map first
     fill_slots_kernel<<<static_cast<unsigned>((pl.n_tok + 255) / 256), 256, 0, st>>>(slot_of_token, pl.n_tok);
-    scatter_slots_kernel<<<static_cast<unsigned>((pl.M + 255) / 256), 256, 0, st>>>(caller_idx, pl.M, slot_of_token, pl.n_tok);
+    if (pl.M > 0 && caller_idx != nullptr)
+      scatter_slots_kernel<<<static_cast<unsigned>((pl.M + 255) / 256), 256, 0, st>>>(caller_idx, pl.M, slot_of_token, pl.n_tok);
     cudaError_t e0 = cudaGetLastError();
     if (e0 != cudaSuccess) return e0;
     idx = nullptr;

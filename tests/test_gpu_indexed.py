@@ -71,6 +71,26 @@ def test_random_subset(diag, mean_fill):
     _check(wl, idx, seed=3)
 
 
+@pytest.mark.parametrize("diag,mean_fill", [(0, 2), (0, 1), (1, 2), (1, 1), (1, 0)])
+def test_nothing_retained_is_the_single_mean_pair_layer(diag, mean_fill):
+    """G2M (Sec. 5.4): no retained keys at all; one mean pair over every token (special tokens included) and,
+    with the diagonal on, the query's own column.  Several query tiles and a ragged tail."""
+    wl = inputs.Workload("g2m", 3, 10, 13, 5, 4, 64, 4, diag, mean_fill, "proj")
+    _check(wl, np.zeros(0, dtype=np.int32), seed=7)
+
+
+def test_nothing_retained_and_no_other_column_is_rejected():
+    wl = inputs.Workload("g2m_none", 2, 4, 4, 5, 2, 64, 4, 0, 0, "iid")
+    params = P.make_params(wl.n_frames, wl.grid_h, wl.grid_w, wl.n_special, wl.n_heads, wl.head_dim, wl.sigma, diag=0, mean_fill=0)
+    Q, K, V = inputs.make_qkv(wl, seed=0, device="cuda")
+    slots = torch.empty((wl.n_tokens,), dtype=torch.int32, device="cuda")
+    ws = torch.empty((1 << 20,), dtype=torch.uint8, device="cuda")
+    with pytest.raises(P.AvggtError) as ei:
+        P.avggt_build_kv_indexed(params, None, 0, K, V, None, None, slots, None, None, ws, ws.numel())
+    assert ei.value.code == -1
+    torch.cuda.synchronize()
+
+
 def test_grid_subset_given_as_a_list_equals_the_grid_layer():
     wl = inputs.Workload("grid_as_list", 4, 12, 12, 5, 8, 64, 4, 1, 2, "proj")
     ocfg = orc.SGAConfig(wl.n_frames, wl.grid_h, wl.grid_w, wl.n_special, wl.n_heads, wl.head_dim, wl.sigma)
