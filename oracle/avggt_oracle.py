@@ -377,3 +377,47 @@ def global_attn_indexed(cfg, idx, Q, K, V, rows=None, return_lse=False):
         lse[out_i] = (mx + np.log(z))[:, 0]
     return (O, lse) if return_lse else O
 
+
+
+def round_to_bf16(x):
+    """Round-to-nearest-even of real values to the bfloat16 grid (returned as float64): the value is first taken
+    to float32, whose upper 16 bits are then rounded (the carry of the lower half, ties to even)."""
+    f = np.ascontiguousarray(np.asarray(x, dtype=np.float32))
+    bits = f.view(np.uint32).astype(np.uint64)
+    lower = bits & 0xFFFF
+    upper = bits >> 16
+    round_up = (lower > 0x8000) | ((lower == 0x8000) & ((upper & 1) == 1))
+    upper = upper + round_up.astype(np.uint64)
+    out = (upper << 16).astype(np.uint32).view(np.float32)
+    out = np.where(np.isfinite(f), out, f)
+    return out.astype(np.float64)
+
+
+def project_build_kv(cfg, X, Wk, Wv, bias_k=None, bias_v=None):
+    """K/V projection followed by the compaction of Sec. 4.3, as one operation (the projection's epilogue does
+    the compaction, so that diagonal preservation and mean-fill cost no second pass over K and V).
+
+    X [N*L, C]; Wk, Wv [H*d, C] (one row per output, as a linear layer stores its weight); biases [H*d] or None.
+    K = X Wk^T + bias_k and V likewise, in float64.  Returns
+      K_b, V_b  [N*L, H, d]: the projections rounded to bfloat16 (what the layer stores and attends to),
+      Kc, Vc    [M, H, d]:   their retained rows, idx [M],
+      kmean, vmean [H, d]:   mean over the dropped patch tokens of the projections BEFORE the rounding
+                             (None when nothing is dropped).
+    """
+    X = np.asarray(X, dtype=np.float64)
+    H, d = cfg.n_heads, cfg.head_dim
+    assert X.shape[0] == cfg.n_tokens and Wk.shape == (H * d, X.shape[1]) and Wv.shape == Wk.shape
+    K = X @ np.asarray(Wk, dtype=np.float64).T
+    V = X @ np.asarray(Wv, dtype=np.float64).T
+    if bias_k is not None:
+        K = K + np.asarray(bias_k, dtype=np.float64)[None, :]
+    if bias_v is not None:
+        V = V + np.asarray(bias_v, dtype=np.float64)[None, :]
+    K = K.reshape(cfg.n_tokens, H, d)
+    V = V.reshape(cfg.n_tokens, H, d)
+    K_b, V_b = round_to_bf16(K), round_to_bf16(V)
+    idx = build_index(cfg)
+    dropped = dropped_token_mask(cfg)
+    kmean = K[dropped].mean(axis=0) if dropped.any() else None
+    vmean = V[dropped].mean(axis=0) if dropped.any() else None
+    return K_b, V_b, K_b[idx], V_b[idx], idx, kmean, vmean

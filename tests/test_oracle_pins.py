@@ -433,3 +433,50 @@ def test_indexed_with_nothing_retained_and_the_diagonal_matches_filled_matrix_br
     D = np.ones(cfg.n_tokens, dtype=bool)
     np.testing.assert_allclose(orc.global_attn_indexed(cfg, np.zeros(0, dtype=np.int64), Q, K, V),
                                _brute_force(cfg, Q, K, V, D=D), rtol=0, atol=1e-12)
+
+
+# --------------------------------------------------------------------------
+# projection with the compaction in its epilogue
+# --------------------------------------------------------------------------
+
+def test_round_to_bf16_matches_the_library_conversion():
+    rng = np.random.default_rng(3)
+    x = np.concatenate([rng.standard_normal(4096) * 10.0 ** rng.integers(-6, 6, 4096),
+                        [0.0, -0.0, 1.0, 1.00390625, 1.01171875, 3.3895313892515355e38, 1e-40]]).astype(np.float32)
+    want = torch.from_numpy(x).bfloat16().float().numpy()
+    np.testing.assert_array_equal(orc.round_to_bf16(x).astype(np.float32), want)
+
+
+def test_projection_with_identity_weights_is_the_plain_compaction():
+    cfg = orc.SGAConfig(3, 4, 5, 2, 2, 8, sigma=4)
+    rng = np.random.default_rng(5)
+    C = cfg.n_heads * cfg.head_dim
+    X = torch.from_numpy(rng.standard_normal((cfg.n_tokens, C))).bfloat16().double().numpy()      # on the bf16 grid already
+    eye = np.eye(C)
+    K_b, V_b, Kc, Vc, idx, kmean, vmean = orc.project_build_kv(cfg, X, eye, 2.0 * eye)
+    Kc_w, Vc_w, idx_w, kmean_w, vmean_w = orc.build_kv(cfg, X.reshape(cfg.n_tokens, cfg.n_heads, cfg.head_dim),
+                                                      2.0 * X.reshape(cfg.n_tokens, cfg.n_heads, cfg.head_dim))
+    np.testing.assert_array_equal(idx, idx_w)
+    np.testing.assert_array_equal(Kc, Kc_w)
+    np.testing.assert_array_equal(Vc, Vc_w)
+    np.testing.assert_allclose(kmean, kmean_w, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(vmean, vmean_w, rtol=0, atol=1e-13)
+
+
+def test_projection_mean_is_the_projected_mean_of_the_dropped_tokens():
+    """Linearity: the mean of the projected keys over D equals the projection of the mean token of D."""
+    cfg = orc.SGAConfig(2, 5, 6, 3, 2, 8, sigma=6)
+    rng = np.random.default_rng(6)
+    C = 24
+    X = rng.standard_normal((cfg.n_tokens, C))
+    Wk, Wv = rng.standard_normal((16, C)), rng.standard_normal((16, C))
+    bk, bv = rng.standard_normal(16), rng.standard_normal(16)
+    K_b, V_b, Kc, Vc, idx, kmean, vmean = orc.project_build_kv(cfg, X, Wk, Wv, bk, bv)
+    xbar = X[_dropped_by_slicing(cfg)].mean(axis=0)
+    np.testing.assert_allclose(kmean.reshape(-1), Wk @ xbar + bk, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(vmean.reshape(-1), Wv @ xbar + bv, rtol=0, atol=1e-12)
+    # the stored projections are the rounded ones, row by row what a plain loop gives
+    i = 7
+    want = np.array([sum(X[i, c] * Wk[o, c] for c in range(C)) + bk[o] for o in range(16)])
+    np.testing.assert_array_equal(K_b[i].reshape(-1), orc.round_to_bf16(want))
+    np.testing.assert_array_equal(Kc, K_b[idx])
