@@ -229,6 +229,33 @@ int avggt_global_attn_shard(const avggt_params* p, int64_t n_kept_total, int64_t
                             void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * The K/V projection with the compaction of avggt_build_kv fused into its epilogue (Sec. 4.3: the
+ * diagonal and mean-fill terms add "only O(N)" work; here that work needs no second pass over K
+ * and V, because every tile of the projection is compacted while it is still on chip):
+ *   K = X Wk^T + bias_k,  V = X Wv^T + bias_v       bf16 operands, fp32 accumulation on the tensor cores
+ *   Kc, Vc, idx   as avggt_build_kv would produce them from the bf16-rounded K and V
+ *   kmean, vmean  mean over the dropped patch tokens of the projections BEFORE the rounding to bf16
+ *                 (fp32; the accumulators are at hand), with a fixed summation order
+ *
+ *   model_dim     C, channels of X: a multiple of 64
+ *   X             device, bf16 [N*L, C]
+ *   Wk, Wv        device, bf16 [H*d, C]  (the layout of a linear layer's weight: one row per output)
+ *   bias_k/_v     device, float [H*d], or NULL
+ *   K, V          device, bf16 [N*L, H, d], written; both NULL when the caller does not need the
+ *                 full arrays (avggt_global_attn reads them only when diag != 0)
+ *   Kc, Vc, idx, kmean, vmean   as for avggt_build_kv
+ *   ws            device scratch of at least the size avggt_project_workspace_bytes returns; it starts
+ *                 with a status block like the attention workspace (avggt_check_status reads it)
+ */
+int avggt_project_workspace_bytes(const avggt_params* p, int32_t model_dim, size_t* ws_bytes);
+int avggt_project_build_kv(const avggt_params* p, int32_t model_dim,
+                           const void* X, const void* Wk, const void* Wv,
+                           const float* bias_k, const float* bias_v,
+                           void* K, void* V, void* Kc, void* Vc, int32_t* idx,
+                           float* kmean, float* vmean,
+                           void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * The exchange step of a frame-sharded run, in two library calls around the caller's two collectives
  * (Sec. 4.3 defines S and the mean pair over all frames, so the ranks exchange their compact K/V and
  * the sums behind the mean once per layer; the library itself does no communication).

@@ -26,7 +26,7 @@ AVGGT_MEAN_OFF, AVGGT_MEAN_UNIT, AVGGT_MEAN_FILL = 0, 1, 2
 EXPORTS = (
     "avggt_kv_count", "avggt_workspace_bytes", "avggt_build_kv", "avggt_build_kv_noalloc", "avggt_global_attn",
     "avggt_frame_attn", "avggt_build_kv_indexed", "avggt_global_attn_indexed", "avggt_global_attn_shard",
-    "avggt_build_kv_shard", "avggt_shard_assemble",
+    "avggt_build_kv_shard", "avggt_shard_assemble", "avggt_project_workspace_bytes", "avggt_project_build_kv",
     "avggt_check_status", "avggt_strerror", "avggt_last_cuda_error", "avggt_version",
 )
 
@@ -81,6 +81,8 @@ def load_library(path):
         "avggt_global_attn_shard": [pp, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp],
         "avggt_build_kv_shard": [pp, vp, vp, vp, i64, vp, vp, vp, sz, vp],
         "avggt_shard_assemble": [pp, vp, ctypes.c_int32, i64p, i64, vp, i64, vp, vp, vp, vp, vp],
+        "avggt_project_workspace_bytes": [pp, ctypes.c_int32, szp],
+        "avggt_project_build_kv": [pp, ctypes.c_int32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp],
         "avggt_check_status": [vp, ctypes.POINTER(ctypes.c_uint32)],
         "avggt_strerror": [ctypes.c_int],
         "avggt_last_cuda_error": [],
@@ -204,6 +206,22 @@ def avggt_shard_assemble(params, gathered, kept, slot_rows, sums, n_dropped_tota
     _check(lib().avggt_shard_assemble(ctypes.byref(params), _ptr(gathered), len(kept), arr, slot_rows, _ptr(sums),
                                       n_dropped_total, _ptr(Kc), _ptr(Vc), _ptr(kmean), _ptr(vmean), stream),
            "avggt_shard_assemble")
+
+
+def avggt_project_workspace_bytes(params, model_dim):
+    """-> workspace bytes of avggt_project_build_kv on the current CUDA device."""
+    b = ctypes.c_size_t()
+    _check(lib().avggt_project_workspace_bytes(ctypes.byref(params), model_dim, ctypes.byref(b)), "avggt_project_workspace_bytes")
+    return b.value
+
+
+def avggt_project_build_kv(params, model_dim, X, Wk, Wv, bias_k, bias_v, K, V, Kc, Vc, idx, kmean, vmean, ws, ws_bytes,
+                           stream=None):
+    """Enqueue K = X Wk^T + bias_k, V = X Wv^T + bias_v with the K/V compaction and the mean reduction in the
+    projection's epilogue.  K, V (the full arrays) may both be None."""
+    _check(lib().avggt_project_build_kv(ctypes.byref(params), model_dim, _ptr(X), _ptr(Wk), _ptr(Wv), _ptr(bias_k),
+                                        _ptr(bias_v), _ptr(K), _ptr(V), _ptr(Kc), _ptr(Vc), _ptr(idx), _ptr(kmean),
+                                        _ptr(vmean), _ptr(ws), ws_bytes, stream), "avggt_project_build_kv")
 
 
 def avggt_frame_attn(params, Q, K, V, O, lse, ws, ws_bytes, stream=None):

@@ -13,7 +13,7 @@ LIB = os.path.join(HERE, "libavggt.so")
 # without hanging or faulting anything.  The product library never contains that switch.
 WAIT_TEST_LIB = os.path.join(HERE, "libavggt_waittest.so")
 WAIT_TEST_DEFINES = ["-DAVGGT_TEST_SKIP_K_LOAD=1", "-DAVGGT_WAIT_LIMIT_NS=500000ull"]
-SOURCES = ["api.cu", "build_kv.cu", "build_kv_noalloc.cu", "global_attn.cu"]
+SOURCES = ["api.cu", "build_kv.cu", "build_kv_noalloc.cu", "global_attn.cu", "project_kv.cu"]
 HEADERS = ["internal.h", "plan.h", "ptx.cuh", "tmap.h", os.path.join("..", "..", "include", "avggt.h")]
 
 

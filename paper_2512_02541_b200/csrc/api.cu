@@ -249,6 +249,43 @@ int avggt_global_attn_shard(const avggt_params* p, int64_t n_kept_total, int64_t
   return run_attn(pl, AttnCall{Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws, ws_bytes, cuda_stream, nullptr, false});
 }
 
+int avggt_project_workspace_bytes(const avggt_params* p, int32_t model_dim, size_t* ws_bytes) {
+  Plan pl;
+  int rc = make_plan(p, &pl);
+  if (rc != AVGGT_OK) return rc;
+  if (model_dim < 64 || model_dim % 64 != 0) return AVGGT_ERR_UNSUPPORTED;
+  DeviceInfo di;
+  rc = device_info(&di);
+  if (rc != AVGGT_OK) return rc;
+  if (ws_bytes) *ws_bytes = project_kv_ws_bytes(pl, di.sm_count);
+  return AVGGT_OK;
+}
+
+int avggt_project_build_kv(const avggt_params* p, int32_t model_dim, const void* X, const void* Wk, const void* Wv,
+                           const float* bias_k, const float* bias_v, void* K, void* V, void* Kc, void* Vc, int32_t* idx,
+                           float* kmean, float* vmean, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Plan pl;
+  int rc = make_plan(p, &pl);
+  if (rc != AVGGT_OK) return rc;
+  if (model_dim < 64 || model_dim % 64 != 0) return AVGGT_ERR_UNSUPPORTED;
+  if (!X || !Wk || !Wv || !Kc || !Vc || !ws) return AVGGT_ERR_INVALID_ARG;
+  if ((K == nullptr) != (V == nullptr)) return AVGGT_ERR_INVALID_ARG;
+  if (pl.mean_fill != 0 && (!kmean || !vmean)) return AVGGT_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(Wk) || !aligned16(Wv) || !aligned16(K) || !aligned16(V) || !aligned16(Kc) ||
+      !aligned16(Vc) || !aligned16(ws) || (reinterpret_cast<uintptr_t>(idx) & 3u) || !aligned16(kmean) ||
+      !aligned16(vmean) || (reinterpret_cast<uintptr_t>(bias_k) & 3u) || (reinterpret_cast<uintptr_t>(bias_v) & 3u))
+    return AVGGT_ERR_ALIGNMENT;
+  DeviceInfo di;
+  rc = device_info(&di);
+  if (rc != AVGGT_OK) return rc;
+  if (ws_bytes < project_kv_ws_bytes(pl, di.sm_count)) return AVGGT_ERR_WORKSPACE_TOO_SMALL;
+  bool tmap_failed = false;
+  const cudaError_t e = launch_project_kv(pl, di.sm_count, model_dim, X, Wk, Wv, bias_k, bias_v, K, V, Kc, Vc, idx, kmean,
+                                          vmean, ws, static_cast<cudaStream_t>(cuda_stream), &tmap_failed);
+  if (tmap_failed) return record_message("cuTensorMapEncodeTiled failed");
+  return record_cuda(e);
+}
+
 int avggt_build_kv_shard(const avggt_params* p, const void* K, const void* V, void* slot, int64_t slot_rows,
                          int32_t* idx, float* sums, void* ws, size_t ws_bytes, void* cuda_stream) {
   Plan pl;

@@ -51,4 +51,12 @@ cudaError_t launch_global_attn(const Plan& pl, int sm_count, const void* Q, cons
 cudaError_t launch_frame_attn(const Plan& pl, const void* Q, const void* K, const void* V, void* O, float* lse, void* ws,
                               cudaStream_t st, bool* tmap_failed);
 
+// ---- K/V projection with the compaction in its epilogue (project_kv.cu)
+size_t project_kv_ws_bytes(const Plan& pl, int sm_count);
+// X [n_tok, model_dim], Wk / Wv [H * d, model_dim] (the layout of a linear layer's weight), bias_k / bias_v [H * d] or
+// null; K / V [n_tok, H, d] or null (written when given); the other outputs as for launch_build_kv.
+cudaError_t launch_project_kv(const Plan& pl, int sm_count, int model_dim, const void* X, const void* Wk, const void* Wv,
+                              const float* bias_k, const float* bias_v, void* K, void* V, void* Kc, void* Vc, int32_t* idx,
+                              float* kmean, float* vmean, void* ws, cudaStream_t st, bool* tmap_failed);
+
 }  // namespace avggt
