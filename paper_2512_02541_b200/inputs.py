@@ -64,6 +64,7 @@ WORKLOADS = {
     # VGGT-shaped layers
     # 30 frames: larger than L2 but small enough for a full profiler capture
     "vggt_n30_s4": _vggt("vggt_n30_s4", 30, 4),
+    "vggt_n30_s9": _vggt("vggt_n30_s9", 30, 9),
     "vggt_n100_s4": _vggt("vggt_n100_s4", 100, 4),
     "vggt_n300_s6": _vggt("vggt_n300_s6", 300, 6),
     "vggt_n800_s9": _vggt("vggt_n800_s9", 800, 9),
