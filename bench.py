@@ -39,13 +39,14 @@ if ROOT not in sys.path:
 from paper_2512_02541_b200 import inputs  # noqa: E402
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
-# profiles/; None where no capture covers the workload.  The attention kernel is captured on the 30-frame copy of
-# the layer (profiles/global_attn_kernel_vggt_n30_s4.md); its traffic is proportional to the frame count, so the
-# 100-frame figure is that capture x 100/30.  The compaction kernel is captured on the 100-frame workload itself.
-_ATTN_N30 = 0.299442e9 + 0.068250e9
+# profiles/; None where no capture covers the workload.  Both kernels are captured on the 30-frame copy of the
+# headline layer (profiles/*_vggt_n30_s9.md); their traffic is proportional to the frame count, so the 800-frame
+# figures are those captures x 800/30.
+_ATTN_N30_S9 = 0.275029760e9 + 0.067800832e9
+_BUILD_N30_S9 = 0.168853760e9 + 0.007183104e9
 NCU_TRAFFIC = {
-    "vggt_n30_s4": {"global_attn_kernel": _ATTN_N30},
-    "vggt_n100_s4": {"global_attn_kernel": _ATTN_N30 * 100 / 30, "build_kv_kernel": 0.562844e9 + 0.103259e9},
+    "vggt_n30_s9": {"global_attn_kernel": _ATTN_N30_S9, "build_kv_kernel": _BUILD_N30_S9},
+    "vggt_n800_s9": {"global_attn_kernel": _ATTN_N30_S9 * 800 / 30, "build_kv_kernel": _BUILD_N30_S9 * 800 / 30},
 }
 
 METRIC = "subsampled_global_attn_queries_per_sec"
