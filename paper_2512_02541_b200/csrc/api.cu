@@ -176,7 +176,7 @@ static int run_attn(const Plan& pl, const AttnCall& c) {
   bool tmap_failed = false;
   const cudaStream_t st = static_cast<cudaStream_t>(c.stream);
   const cudaError_t e = c.frame_mode
-      ? launch_frame_attn(pl, c.Q, c.K, c.V, c.O, c.lse, c.ws, st, &tmap_failed)
+      ? launch_frame_attn(pl, di.sm_count, c.Q, c.K, c.V, c.O, c.lse, c.ws, st, &tmap_failed)
       : launch_global_attn(pl, di.sm_count, c.Q, c.K, c.V, c.Kc, c.Vc, c.kmean, c.vmean, c.O, c.lse, c.ws, st,
                            &tmap_failed, c.slot_of_token);
   if (tmap_failed) return record_message("cuTensorMapEncodeTiled failed");

@@ -83,13 +83,18 @@ struct AttnArgs {
                         //    blockIdx.z is the frame, keys and values are the frame's own rows of K and V
   int64_t n_keys;       // keys of one problem: M, or the tokens of a frame
   int32_t n_kv_tiles;   // ceil(n_keys / 128)
+  int32_t n_work;       // work items (pairs of query tiles x heads x problems) of the launch; a CTA takes the items
+                        // blockIdx.x, blockIdx.x + gridDim.x, ...  (more than one per CTA only in frame attention)
+  int32_t pairs;        // pairs of query tiles of one problem
   int32_t use_diag;     // diag on and |D| > 0
   int32_t use_mean;     // mean_fill on and |D| > 0
   float scale_log2;     // softmax scale * log2(e)
 };
 
 struct __align__(8) Barriers {
-  uint64_t q_full;
+  uint64_t q_full;             // producer -> all: the work item's Q tiles are in shared memory
+  uint64_t q_empty;            // MMA issuers -> producer: every Q K^T of the work item has completed, Q may be overwritten
+  uint64_t o_free[kQTiles];    // softmax -> MMA: O_t of the finished work item has been read out
   uint64_t k_full[kStages], k_empty[kStages];
   uint64_t v_full[kStages], v_empty[kStages];
   uint64_t s_full[kQTiles];    // MMA -> softmax: S_t(j) is in tensor memory
@@ -105,7 +110,7 @@ struct __align__(8) Barriers {
 
 __device__ __forceinline__ void report_timeout(const AttnArgs& a, Barriers* bars, uint32_t where, uint32_t iter) {
   if (atomicCAS(a.status, 0u, 1u) == 0u) {
-    a.status[1] = blockIdx.x + (blockIdx.y + blockIdx.z * gridDim.y) * gridDim.x;
+    a.status[1] = blockIdx.x;
     a.status[2] = where;
     a.status[3] = iter;
   }
@@ -171,6 +176,25 @@ struct CtaProblem {
   int key_row0;       // frame attention: token index of the frame's first key
 };
 
+// Work item -> problem.  Items are numbered with the pair of query tiles fastest, then the head, then (frame
+// attention) the frame, so that the CTAs running side by side share one head's keys in L2.
+__device__ __forceinline__ CtaProblem work_item(const AttnArgs& a, int item) {
+  CtaProblem c;
+  const int qp = item % a.pairs;
+  const int rest = item / a.pairs;
+  c.head = rest % a.pl.H;
+  if (a.frame_mode) {
+    c.key_row0 = (rest / a.pl.H) * a.pl.L;
+    c.q0 = c.key_row0 + qp * (kQTiles * kTileQ);
+    c.row_end = static_cast<int64_t>(c.key_row0) + a.pl.L;
+  } else {
+    c.key_row0 = 0;
+    c.q0 = qp * (kQTiles * kTileQ);
+    c.row_end = a.pl.n_tok;
+  }
+  return c;
+}
+
 struct SmemLayout {
   uint8_t* q[kQTiles];
   uint8_t* k;   // kStages tiles
@@ -191,61 +215,73 @@ __device__ __forceinline__ bool wait_bar_warp(uint64_t* bar, uint32_t parity, Ba
 // ------------------------------------------------------------------ TMA producer (one warp)
 __device__ __forceinline__ void producer_role(const CUtensorMap* tm_q, const CUtensorMap* tm_k, const CUtensorMap* tm_v,
                                               const CUtensorMap* tm_kc, const CUtensorMap* tm_vc, const AttnArgs& a,
-                                              Barriers* bars, const SmemLayout& sm, const CtaProblem& cta) {
+                                              Barriers* bars, const SmemLayout& sm) {
   const int n_kv = a.n_kv_tiles;
-  const int n_items = n_kv + (a.use_diag ? kQTiles : 0);
-  const int head = cta.head, q0 = cta.q0;
+  const int n_ring = n_kv + (a.use_diag ? kQTiles : 0);   // ring items of one work item
   if (elect_one()) {
     prefetch_tensormap(tm_q);
     prefetch_tensormap(tm_kc);
     prefetch_tensormap(tm_vc);
-    mbar_arrive_expect_tx(smem_u32(&bars->q_full), kQTiles * kTileBytes);
-#pragma unroll
-    for (int t = 0; t < kQTiles; ++t)
-      tma_load_2d(smem_u32(sm.q[t]), tm_q, head * kHeadDim, q0 + t * kTileQ, smem_u32(&bars->q_full));
   }
-  __syncwarp();
-  int it = 0;
-  int k_issued = 0, v_issued = 0;   // ring items whose K / V copy has been issued
+  int k_issued = 0, v_issued = 0;   // K / V copies issued so far, over all work items
   int stage = 0;
   uint32_t empty_parity = 1;   // a fresh barrier passes the wait on the "previous" phase at once
   bool ok = true;
-  for (; it < n_items; ++it) {
-    ok = wait_bar_warp(&bars->k_empty[stage], empty_parity, bars, a, 10, it);
-    if (!ok) break;
-#ifdef AVGGT_TEST_SKIP_K_LOAD
-    // Build for the wait-limit test only (never part of libavggt.so): the first thread block leaves out one K
-    // tile, so that the waits on it run out, the block reports the time-out and every role leaves in order.
-    const bool skip_load = it == AVGGT_TEST_SKIP_K_LOAD && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0;
-#else
-    constexpr bool skip_load = false;
-#endif
-    if (elect_one() && !skip_load) {
-      const uint32_t kb = smem_u32(&bars->k_full[stage]);
-      mbar_arrive_expect_tx(kb, kTileBytes);
-      if (a.frame_mode) tma_load_2d(smem_u32(sm.k + stage * kTileBytes), tm_k, head * kHeadDim, cta.key_row0 + it * kTileKV, kb);
-      else if (it < n_kv) tma_load_3d(smem_u32(sm.k + stage * kTileBytes), tm_kc, 0, it * kTileKV, head, kb);
-      else tma_load_2d(smem_u32(sm.k + stage * kTileBytes), tm_k, head * kHeadDim, q0 + (it - n_kv) * kTileQ, kb);
+  int n_done = 0;              // work items completed by this role
+  int q_issued = 0;            // work items whose Q copies have been issued
+  for (int item = blockIdx.x; item < a.n_work && ok; item += gridDim.x, ++n_done) {
+    const CtaProblem cta = work_item(a, item);
+    const int head = cta.head, q0 = cta.q0;
+    // the Q tiles of the previous work item are no longer read by any Q K^T
+    if (n_done > 0) {
+      ok = wait_bar_warp(&bars->q_empty, (n_done - 1) & 1, bars, a, 14, n_done);
+      if (!ok) break;
     }
-    __syncwarp();
-    k_issued = it + 1;
-    ok = wait_bar_warp(&bars->v_empty[stage], empty_parity, bars, a, 11, it);
-    if (!ok) break;
     if (elect_one()) {
-      const uint32_t vb = smem_u32(&bars->v_full[stage]);
-      mbar_arrive_expect_tx(vb, kTileBytes);
-      if (a.frame_mode) tma_load_2d(smem_u32(sm.v + stage * kTileBytes), tm_v, head * kHeadDim, cta.key_row0 + it * kTileKV, vb);
-      else if (it < n_kv) tma_load_3d(smem_u32(sm.v + stage * kTileBytes), tm_vc, 0, it * kTileKV, head, vb);
-      else tma_load_2d(smem_u32(sm.v + stage * kTileBytes), tm_v, head * kHeadDim, q0 + (it - n_kv) * kTileQ, vb);
+      mbar_arrive_expect_tx(smem_u32(&bars->q_full), kQTiles * kTileBytes);
+#pragma unroll
+      for (int t = 0; t < kQTiles; ++t)
+        tma_load_2d(smem_u32(sm.q[t]), tm_q, head * kHeadDim, q0 + t * kTileQ, smem_u32(&bars->q_full));
     }
     __syncwarp();
-    v_issued = it + 1;
-    if (++stage == kStages) { stage = 0; empty_parity ^= 1; }
+    ++q_issued;
+    for (int it = 0; it < n_ring; ++it) {
+      ok = wait_bar_warp(&bars->k_empty[stage], empty_parity, bars, a, 10, it);
+      if (!ok) break;
+#ifdef AVGGT_TEST_SKIP_K_LOAD
+      // Build for the wait-limit test only (never part of libavggt.so): the first thread block leaves out one K
+      // tile, so that the waits on it run out, the block reports the time-out and every role leaves in order.
+      const bool skip_load = it == AVGGT_TEST_SKIP_K_LOAD && n_done == 0 && blockIdx.x == 0;
+#else
+      constexpr bool skip_load = false;
+#endif
+      if (elect_one() && !skip_load) {
+        const uint32_t kb = smem_u32(&bars->k_full[stage]);
+        mbar_arrive_expect_tx(kb, kTileBytes);
+        if (a.frame_mode) tma_load_2d(smem_u32(sm.k + stage * kTileBytes), tm_k, head * kHeadDim, cta.key_row0 + it * kTileKV, kb);
+        else if (it < n_kv) tma_load_3d(smem_u32(sm.k + stage * kTileBytes), tm_kc, 0, it * kTileKV, head, kb);
+        else tma_load_2d(smem_u32(sm.k + stage * kTileBytes), tm_k, head * kHeadDim, q0 + (it - n_kv) * kTileQ, kb);
+      }
+      __syncwarp();
+      ++k_issued;
+      ok = wait_bar_warp(&bars->v_empty[stage], empty_parity, bars, a, 11, it);
+      if (!ok) break;
+      if (elect_one()) {
+        const uint32_t vb = smem_u32(&bars->v_full[stage]);
+        mbar_arrive_expect_tx(vb, kTileBytes);
+        if (a.frame_mode) tma_load_2d(smem_u32(sm.v + stage * kTileBytes), tm_v, head * kHeadDim, cta.key_row0 + it * kTileKV, vb);
+        else if (it < n_kv) tma_load_3d(smem_u32(sm.v + stage * kTileBytes), tm_vc, 0, it * kTileKV, head, vb);
+        else tma_load_2d(smem_u32(sm.v + stage * kTileBytes), tm_v, head * kHeadDim, q0 + (it - n_kv) * kTileQ, vb);
+      }
+      __syncwarp();
+      ++v_issued;
+      if (++stage == kStages) { stage = 0; empty_parity ^= 1; }
+    }
   }
   if (!ok) {
-    // let the copies still in flight land before the CTA gives up its shared memory: the last kStages
-    // issued into either ring (earlier ones completed before their stage was reused)
-    (void)wait_bar_warp(&bars->q_full, 0, bars, a, 12, 0, false);
+    // let the copies still in flight land before the CTA gives up its shared memory: the Q tiles of the last work
+    // item begun, and the last kStages issued into either ring (earlier ones completed before their stage was reused)
+    if (q_issued > 0) (void)wait_bar_warp(&bars->q_full, (q_issued - 1) & 1, bars, a, 12, 0, false);
     for (int back = 1; back <= kStages; ++back) {
       const int jk = k_issued - back, jv = v_issued - back;
       if (jk >= 0) (void)wait_bar_warp(&bars->k_full[jk % kStages], (jk / kStages) & 1, bars, a, 12, jk, false);
@@ -296,28 +332,50 @@ __device__ __forceinline__ void mma_issue_loop(const AttnArgs& a, Barriers* bars
   const int n_kv = a.n_kv_tiles;
   const uint64_t desc_q = umma_desc_sw128(smem_u32(sm.q[t]));
   const uint32_t k_base = smem_u32(sm.k), v_base = smem_u32(sm.v);
-
   if (n_kv == 0) return;   // no retained keys: the epilogue's two extra columns are the whole layer
-  if (!wait_bar_warp(&bars->q_full, 0, bars, a, 20, 0)) return;
-  if (!wait_bar_warp(&bars->k_full[0], 0, bars, a, 21, 0)) return;
-  tc_fence_after();
-  issue_qk<t>(a, bars, tmem, desc_q, k_base, 0, 0);
 
-  int k_stage = 1, v_stage = 0;          // stage of K_{j+1} and of V_j
+  // Running over all work items of the CTA: the ring positions of the next K and V tile, and g, the number of key
+  // steps of this tile so far (the phase of the per-step barriers).  The rings carry the work item's own rows
+  // (the diagonal) only in the subsampled layer, where a CTA has one work item.
+  int k_stage = 0, v_stage = 0;
   uint32_t k_parity = 0, v_parity = 0;   // parity of their "full" phase
-  for (int j = 0; j < n_kv; ++j) {
-    if (j + 1 < n_kv) {
-      if (!wait_bar_warp(&bars->s_free[t], j & 1, bars, a, 22 + t, j)) return;
-      if (!wait_bar_warp(&bars->k_full[k_stage], k_parity, bars, a, 24 + t, j)) return;
-      tc_fence_after();
-      issue_qk<t>(a, bars, tmem, desc_q, k_base, k_stage, j + 1);
-      if (++k_stage == kStages) { k_stage = 0; k_parity ^= 1; }
-    }
-    if (!wait_bar_warp(&bars->p_full[t], j & 1, bars, a, 26 + t, j)) return;
-    if (!wait_bar_warp(&bars->v_full[v_stage], v_parity, bars, a, 28 + t, j)) return;
+  int g = 0;
+  int n_done = 0;
+  for (int item = blockIdx.x; item < a.n_work; item += gridDim.x, ++n_done, g += n_kv) {
+    if (!wait_bar_warp(&bars->q_full, n_done & 1, bars, a, 20, n_done)) return;
+    // first product of the work item: S_t must have been read by the softmax of the previous item's last step
+    if (n_done > 0 && !wait_bar_warp(&bars->s_free[t], (g - 1) & 1, bars, a, 22 + t, g - 1)) return;
+    if (!wait_bar_warp(&bars->k_full[k_stage], k_parity, bars, a, 21, g)) return;
     tc_fence_after();
-    issue_pv<t>(a, bars, tmem, v_base, v_stage, j);
-    if (++v_stage == kStages) { v_stage = 0; v_parity ^= 1; }
+    issue_qk<t>(a, bars, tmem, desc_q, k_base, k_stage, 0);
+    if (++k_stage == kStages) { k_stage = 0; k_parity ^= 1; }
+    for (int j = 0; j < n_kv; ++j) {
+      if (j + 1 < n_kv) {
+        if (!wait_bar_warp(&bars->s_free[t], (g + j) & 1, bars, a, 22 + t, g + j)) return;
+        if (!wait_bar_warp(&bars->k_full[k_stage], k_parity, bars, a, 24 + t, g + j)) return;
+        tc_fence_after();
+        issue_qk<t>(a, bars, tmem, desc_q, k_base, k_stage, j + 1);
+        if (++k_stage == kStages) { k_stage = 0; k_parity ^= 1; }
+      } else {
+        // every Q K^T of this work item has been issued: when they have completed, Q may be overwritten
+        if (elect_one()) umma_commit(smem_u32(&bars->q_empty));
+        __syncwarp();
+      }
+      if (!wait_bar_warp(&bars->p_full[t], (g + j) & 1, bars, a, 26 + t, g + j)) return;
+      if (!wait_bar_warp(&bars->v_full[v_stage], v_parity, bars, a, 28 + t, g + j)) return;
+      // the first P V of a work item overwrites O_t: the previous item's epilogue must have read it out
+      if (j == 0 && n_done > 0 && !wait_bar_warp(&bars->o_free[t], (n_done - 1) & 1, bars, a, 29, n_done)) return;
+      tc_fence_after();
+      issue_pv<t>(a, bars, tmem, v_base, v_stage, j);
+      if (++v_stage == kStages) { v_stage = 0; v_parity ^= 1; }
+    }
+    // ring positions of the work item's own K/V rows (read by the softmax epilogue, not by any product)
+    if (a.use_diag) {
+      for (int i = 0; i < kQTiles; ++i) {
+        if (++k_stage == kStages) { k_stage = 0; k_parity ^= 1; }
+        if (++v_stage == kStages) { v_stage = 0; v_parity ^= 1; }
+      }
+    }
   }
 }
 
@@ -423,13 +481,15 @@ __device__ __forceinline__ bool pair_sync(uint32_t phase, const SoftmaxThread& m
 // released, so that the next Q K^T runs under this step's exponentials.  The row maximum (of both
 // halves, exchanged with the partner thread) decides whether the reference maximum moves (lazy
 // rescale); both threads of a row take the same decision from the same numbers.
-// kPoly: pairs per eight whose exponential is a polynomial.  kLse: also keep the sum of the
+// j: step within the work item; g: the tile's steps in the CTA's earlier work items; pair_phase: meetings with
+// the partner thread so far.  kPoly: pairs per eight whose exponential is a polynomial.  kLse: also keep the sum of the
 // unrounded exponentials, for the log-sum-exp output.  kMasked: columns >= valid are excluded
 // (valid counts from this thread's first column and may be <= 0).
 template <bool kMasked, bool kLse, int kPoly>
-__device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int valid, float scale_log2, float& m_used,
-                                             float& l_run, float& l_exact, Barriers* bars, PairExchange* px,
-                                             const AttnArgs& a) {
+__device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int g, uint32_t pair_phase, int valid,
+                                             float scale_log2, float& m_used, float& l_run, float& l_exact, Barriers* bars,
+                                             PairExchange* px, const AttnArgs& a) {
+  const int gj = g + j;   // this tile's key steps so far, over all work items of the CTA: the phase of the per-step barriers
   uint32_t s[64];
   {
     uint32_t (&s2)[2][32] = reinterpret_cast<uint32_t (&)[2][32]>(s);
@@ -455,9 +515,9 @@ __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int
   }
   const float half_max = fmaxf(mx[0], mx[1]);
   // two slots, by step parity: the partner may still be reading the previous step's value
-  px->step[me.t][j & 1][me.h][me.r] = half_max;
-  if (!pair_sync(static_cast<uint32_t>(j), me, bars, a)) return false;
-  const float other_max = *reinterpret_cast<const volatile float*>(&px->step[me.t][j & 1][me.h ^ 1][me.r]);
+  px->step[me.t][gj & 1][me.h][me.r] = half_max;
+  if (!pair_sync(pair_phase, me, bars, a)) return false;
+  const float other_max = *reinterpret_cast<const volatile float*>(&px->step[me.t][gj & 1][me.h ^ 1][me.r]);
   const float tile_max = fmaxf(half_max, other_max) * scale_log2;
   // lazy rescale: keep the old reference maximum unless the new one is far above it
   const bool jump = tile_max > m_used + kRescaleThreshold;
@@ -472,7 +532,7 @@ __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int
 
   // P_t(j-1) must have been consumed, and O_t be at rest, before either is written
   if (j > 0) {
-    if (!wait_bar(&bars->o_done[me.t], (j - 1) & 1, bars, a, 30 + me.t, j)) return false;
+    if (!wait_bar(&bars->o_done[me.t], (gj - 1) & 1, bars, a, 30 + me.t, gj)) return false;
     tc_fence_after();
   }
   if (rescale) {   // this thread's 32 of the row's 64 accumulator columns
@@ -485,7 +545,7 @@ __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int
   }
 #if AVGGT_PINGPONG
   // this tile's turn on the exponential unit: the other tile's two warps on this scheduler have left their phase
-  if (!wait_bar(&bars->turn[me.t][me.q], j & 1, bars, a, 62 + me.t, j)) return false;
+  if (!wait_bar(&bars->turn[me.t][me.q], gj & 1, bars, a, 62 + me.t, gj)) return false;
 #endif
 
   // exponentials, rounded to bf16 for the value product; the normaliser sums the
@@ -513,42 +573,30 @@ __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int
   return true;
 }
 
-__device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, PairExchange* px, const SmemLayout& sm,
-                                             uint32_t tmem, int warp, int lane, const CtaProblem& cta) {
+// One work item of a softmax thread: the key steps, then the epilogue.  g: this tile's key steps in the CTA's earlier
+// work items; pair_phase: meetings with the partner thread so far; n_done: work items before this one.
+__device__ __forceinline__ bool softmax_item(const AttnArgs& a, Barriers* bars, PairExchange* px, const SmemLayout& sm,
+                                             const SoftmaxThread& me, const CtaProblem& cta, int g, uint32_t pair_phase,
+                                             int n_done) {
   const Plan& pl = a.pl;
   const int n_kv = a.n_kv_tiles;
-  SoftmaxThread me;
-  me.t = warp >> 3;
-  me.h = (warp >> 2) & 1;
-  me.q = warp & 3;
-  me.lane = lane;
-  me.r = 32 * me.q + lane;
-  const uint32_t tile_base = tmem + me.t * kTmemTileStride + (static_cast<uint32_t>(32 * me.q) << 16);   // TMEM lane = row
-  me.tS = tile_base + 64 * me.h;
-  me.tP = tile_base + kColP + 32 * me.h;
-  me.tO = tile_base + kColO + 32 * me.h;
-  const int t = me.t, r = me.r;
+  const int t = me.t, r = me.r, lane = me.lane;
   float m_used = -INFINITY;   // reference maximum of the stored exponentials (log2 units); the same in both threads of a row
   float l_run = 0.f;          // this half's sum of the bf16-rounded 2^(scale_log2 * s - m_used): normaliser of O
   float l_exact = 0.f;        // the same sum without the rounding: log-sum-exp output only
   const bool want_lse = a.lse != nullptr;
-#if AVGGT_PINGPONG
-  // tile 0 goes first: tile 1 hands it the first turn
-  if (t == 1 && lane == 0) mbar_arrive(smem_u32(&bars->turn[0][me.q]));
-#endif
-
 #pragma unroll 1
   for (int j = 0; j < n_kv; ++j) {
-    if (!wait_bar(&bars->s_full[t], j & 1, bars, a, 40 + t, j)) return;
+    if (!wait_bar(&bars->s_full[t], (g + j) & 1, bars, a, 40 + t, g + j)) return false;
     tc_fence_after();
     const int valid_tile = static_cast<int>(a.n_keys - static_cast<int64_t>(j) * kTileKV);
     const int valid = valid_tile - 64 * me.h;
     bool ok;
     // the masked (last, ragged) tile keeps every exponential on the special-function unit, where -inf gives an exact 0
-    if (valid_tile < kTileKV) ok = softmax_step<true, true, 0>(me, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a);
-    else if (want_lse) ok = softmax_step<false, true, kPolyEighths>(me, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a);
-    else ok = softmax_step<false, false, kPolyEighths>(me, j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a);
-    if (!ok) return;
+    if (valid_tile < kTileKV) ok = softmax_step<true, true, 0>(me, j, g, pair_phase + j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a);
+    else if (want_lse) ok = softmax_step<false, true, kPolyEighths>(me, j, g, pair_phase + j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a);
+    else ok = softmax_step<false, false, kPolyEighths>(me, j, g, pair_phase + j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a);
+    if (!ok) return false;
   }
 
   // ---- epilogue: diagonal and mean-fill terms, normalisation, store of this thread's 32 output dimensions
@@ -563,24 +611,26 @@ __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, 
   // the row's sums: mine plus the partner's
   px->final[t][0][me.h][r] = l_run;
   px->final[t][1][me.h][r] = l_exact;
-  if (!pair_sync(static_cast<uint32_t>(n_kv), me, bars, a)) return;
+  if (!pair_sync(pair_phase + n_kv, me, bars, a)) return false;
   const float other_run = *reinterpret_cast<const volatile float*>(&px->final[t][0][me.h ^ 1][r]);
   const float other_exact = *reinterpret_cast<const volatile float*>(&px->final[t][1][me.h ^ 1][r]);
   l_run += other_run;
   l_exact += other_exact;
 
   if (n_kv > 0) {
-    if (!wait_bar(&bars->o_done[t], (n_kv - 1) & 1, bars, a, 50 + t, n_kv)) return;
+    if (!wait_bar(&bars->o_done[t], (g + n_kv - 1) & 1, bars, a, 50 + t, g + n_kv)) return false;
     tc_fence_after();
   }
-  if (!wait_bar(&bars->q_full, 0, bars, a, 52, 0)) return;   // completed long ago: makes the Q tile visible to this thread
+  // completed long ago: makes the Q tile visible to this thread.  Only the two extra columns read Q here, and a CTA
+  // that has them has one work item (a later item's Q may already be on its way otherwise).
+  if ((a.use_diag || a.use_mean) && !wait_bar(&bars->q_full, n_done & 1, bars, a, 52, 0)) return false;
   const int item = n_kv + t;                         // ring item holding this tile's own K/V rows
   const uint8_t* sKd = sm.k + (item % kStages) * kTileBytes;
   const uint8_t* sVd = sm.v + (item % kStages) * kTileBytes;
   if (a.use_diag) {
     const uint32_t par = (item / kStages) & 1;
-    if (!wait_bar(&bars->k_full[item % kStages], par, bars, a, 53, item)) return;
-    if (!wait_bar(&bars->v_full[item % kStages], par, bars, a, 54, item)) return;
+    if (!wait_bar(&bars->k_full[item % kStages], par, bars, a, 53, item)) return false;
+    if (!wait_bar(&bars->v_full[item % kStages], par, bars, a, 54, item)) return false;
   }
   const uint8_t* sQ = sm.q[t];
   // base-2 logits of the two extra columns; both threads of a row compute them in full, from the same numbers
@@ -624,6 +674,10 @@ __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, 
   if (n_kv > 0) {
     tmem_ld32(me.tO, o);
     tmem_wait_ld();
+    // O_t is in registers: the next work item's first P V may overwrite it
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&bars->o_free[t]));
   } else {   // no retained keys at all: the accumulator was never written
 #pragma unroll
     for (int i = 0; i < 32; ++i) o[i] = 0u;
@@ -662,6 +716,35 @@ __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, 
       a.lse[static_cast<size_t>(row) * pl.H + head] = (m_fin + log2f(z_exact)) * 0.6931471805599453f;
     }
   }
+  return true;
+}
+
+__device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, PairExchange* px, const SmemLayout& sm,
+                                             uint32_t tmem, int warp, int lane) {
+  SoftmaxThread me;
+  me.t = warp >> 3;
+  me.h = (warp >> 2) & 1;
+  me.q = warp & 3;
+  me.lane = lane;
+  me.r = 32 * me.q + lane;
+  const uint32_t tile_base = tmem + me.t * kTmemTileStride + (static_cast<uint32_t>(32 * me.q) << 16);   // TMEM lane = row
+  me.tS = tile_base + 64 * me.h;
+  me.tP = tile_base + kColP + 32 * me.h;
+  me.tO = tile_base + kColO + 32 * me.h;
+#if AVGGT_PINGPONG
+  // tile 0 goes first: tile 1 hands it the first turn
+  if (me.t == 1 && lane == 0) mbar_arrive(smem_u32(&bars->turn[0][me.q]));
+#endif
+  const int n_kv = a.n_kv_tiles;
+  int g = 0, n_done = 0;
+  uint32_t pair_phase = 0;
+#pragma unroll 1
+  for (int item = blockIdx.x; item < a.n_work; item += gridDim.x) {
+    if (!softmax_item(a, bars, px, sm, me, work_item(a, item), g, pair_phase, n_done)) return;
+    g += n_kv;
+    pair_phase += static_cast<uint32_t>(n_kv) + 1u;   // one meeting per step and one in the epilogue
+    ++n_done;
+  }
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -680,23 +763,12 @@ global_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
   const int tid = threadIdx.x;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // warp-uniform by construction
-  CtaProblem cta;
-  cta.head = blockIdx.y;
-  if (a.frame_mode) {
-    cta.key_row0 = static_cast<int>(blockIdx.z) * a.pl.L;
-    cta.q0 = cta.key_row0 + blockIdx.x * (kQTiles * kTileQ);
-    cta.row_end = static_cast<int64_t>(cta.key_row0) + a.pl.L;
-  } else {
-    cta.key_row0 = 0;
-    cta.q0 = blockIdx.x * (kQTiles * kTileQ);
-    cta.row_end = a.pl.n_tok;
-  }
-
   // a launch in which a wait has already run out is abandoned: the remaining CTAs leave at once
   if (__syncthreads_or(*reinterpret_cast<volatile uint32_t*>(a.status) != 0u)) return;
 
   if (tid == 0) {
     mbar_init(smem_u32(&bars.q_full), 1);
+    mbar_init(smem_u32(&bars.q_empty), kQTiles);
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&bars.k_full[s]), 1);
       mbar_init(smem_u32(&bars.k_empty[s]), kQTiles);
@@ -711,6 +783,7 @@ global_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       for (int w = 0; w < 4; ++w) mbar_init(smem_u32(&bars.pair[t][w]), 2);
       for (int w = 0; w < 4; ++w) mbar_init(smem_u32(&bars.turn[t][w]), 2);
       mbar_init(smem_u32(&bars.mma_idle[t]), 1);
+      mbar_init(smem_u32(&bars.o_free[t]), kSoftmaxWarps / kQTiles);
     }
     bars.abort_flag = 0;
     fence_mbar_init();
@@ -726,10 +799,10 @@ global_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
   if (warp < kSoftmaxWarps) {
     reg_inc<kRegsSoftmax>();
-    softmax_role(a, &bars, &pair_exchange, sm, tmem, warp, tid & 31, cta);
+    softmax_role(a, &bars, &pair_exchange, sm, tmem, warp, tid & 31);
   } else {
     reg_dec<kRegsOther>();
-    if (warp == kTmaWarp) producer_role(&tm_q, &tm_k, &tm_v, &tm_kc, &tm_vc, a, &bars, sm, cta);
+    if (warp == kTmaWarp) producer_role(&tm_q, &tm_k, &tm_v, &tm_kc, &tm_vc, a, &bars, sm);
     else if (warp == kMmaWarp) mma_role<0>(a, &bars, sm, tmem);
     else if (warp == kMmaWarp + 1) mma_role<1>(a, &bars, sm, tmem);
   }
@@ -775,7 +848,7 @@ cudaError_t prepare_kernel() {
 }
 
 // Tensor maps and launch shared by the two entry points.  frame_mode: see AttnArgs.
-cudaError_t launch_attn(const Plan& pl, bool frame_mode, const void* Q, const void* K, const void* V, const void* Kc,
+cudaError_t launch_attn(const Plan& pl, int sm_count, bool frame_mode, const void* Q, const void* K, const void* V, const void* Kc,
                         const void* Vc, const float* kmean, const float* vmean, void* O, float* lse, void* ws,
                         cudaStream_t st, bool* tmap_failed, const int32_t* slot_of_token) {
   *tmap_failed = false;
@@ -793,6 +866,9 @@ cudaError_t launch_attn(const Plan& pl, bool frame_mode, const void* Q, const vo
   a.use_diag = (!frame_mode && pl.diag != 0 && pl.n_dropped > 0) ? 1 : 0;
   a.use_mean = (!frame_mode && pl.mean_fill != 0 && pl.n_dropped > 0) ? 1 : 0;
   a.scale_log2 = pl.scale * kLog2e;
+  const int64_t rows = frame_mode ? pl.L : pl.n_tok;
+  a.pairs = static_cast<int32_t>((rows + kQTiles * kTileQ - 1) / (kQTiles * kTileQ));
+  a.n_work = a.pairs * pl.H * (frame_mode ? pl.n_frames : 1);
 
   // token-major [n_tok, H*d] maps for Q and for K, V (the diagonal tiles; all tiles of frame attention);
   // head-major [H, M, d] maps for Kc, Vc
@@ -820,25 +896,26 @@ cudaError_t launch_attn(const Plan& pl, bool frame_mode, const void* Q, const vo
   if (e != cudaSuccess) return e;
   e = cudaMemsetAsync(ws, 0, kAttnStatusBytes, st);
   if (e != cudaSuccess) return e;
-  const int rows_per_cta = kQTiles * kTileQ;
-  const int64_t rows = frame_mode ? pl.L : pl.n_tok;
-  const dim3 grid(static_cast<unsigned>((rows + rows_per_cta - 1) / rows_per_cta), static_cast<unsigned>(pl.H),
-                  frame_mode ? static_cast<unsigned>(pl.n_frames) : 1u);
+  // The subsampled layer: one work item per CTA (hundreds of key steps each).  Frame attention: a dozen key steps
+  // per work item, so one CTA per SM walks over many of them and the next item's loads and first product run
+  // under the current item's epilogue.
+  const unsigned grid = frame_mode ? static_cast<unsigned>(a.n_work < sm_count ? a.n_work : sm_count)
+                                   : static_cast<unsigned>(a.n_work);
   global_attn_kernel<<<grid, kThreads, kAttnSmemBytes, st>>>(tm_q, tm_k, tm_v, tm_kc, tm_vc, a);
   return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_global_attn(const Plan& pl, int /*sm_count*/, const void* Q, const void* K, const void* V,
+cudaError_t launch_global_attn(const Plan& pl, int sm_count, const void* Q, const void* K, const void* V,
                                const void* Kc, const void* Vc, const float* kmean, const float* vmean, void* O,
                                float* lse, void* ws, cudaStream_t st, bool* tmap_failed, const int32_t* slot_of_token) {
-  return launch_attn(pl, false, Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws, st, tmap_failed, slot_of_token);
+  return launch_attn(pl, sm_count, false, Q, K, V, Kc, Vc, kmean, vmean, O, lse, ws, st, tmap_failed, slot_of_token);
 }
 
-cudaError_t launch_frame_attn(const Plan& pl, const void* Q, const void* K, const void* V, void* O, float* lse, void* ws,
-                              cudaStream_t st, bool* tmap_failed) {
-  return launch_attn(pl, true, Q, K, V, nullptr, nullptr, nullptr, nullptr, O, lse, ws, st, tmap_failed, nullptr);
+cudaError_t launch_frame_attn(const Plan& pl, int sm_count, const void* Q, const void* K, const void* V, void* O, float* lse,
+                              void* ws, cudaStream_t st, bool* tmap_failed) {
+  return launch_attn(pl, sm_count, true, Q, K, V, nullptr, nullptr, nullptr, nullptr, O, lse, ws, st, tmap_failed, nullptr);
 }
 
 }  // namespace avggt

@@ -48,8 +48,8 @@ cudaError_t launch_global_attn(const Plan& pl, int sm_count, const void* Q, cons
                                const int32_t* slot_of_token = nullptr);
 
 // Frame attention (Sec. 4.2): the same kernel, one independent dense problem per frame.
-cudaError_t launch_frame_attn(const Plan& pl, const void* Q, const void* K, const void* V, void* O, float* lse, void* ws,
-                              cudaStream_t st, bool* tmap_failed);
+cudaError_t launch_frame_attn(const Plan& pl, int sm_count, const void* Q, const void* K, const void* V, void* O, float* lse,
+                              void* ws, cudaStream_t st, bool* tmap_failed);
 
 // ---- K/V projection with the compaction in its epilogue (project_kv.cu)
 size_t project_kv_ws_bytes(const Plan& pl, int sm_count);
