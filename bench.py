@@ -423,12 +423,16 @@ def run_ours(args, wl):
     e2e_steps = max(1, min(args.steps, 3))
     hQ, hK, hV = (t.cpu().pin_memory() for t in (Q, K, V))
     hO = torch.empty_like(hQ).pin_memory()
-    dQ, dK, dV = (torch.empty_like(t) for t in (Q, K, V))
+    dQ, dK, dV = (torch.empty_like(t) for t in (Q, K, V)) if shard_mode else (None, None, None)
 
     def e2e_step():
-        dQ.copy_(hQ, non_blocking=True); dK.copy_(hK, non_blocking=True); dV.copy_(hV, non_blocking=True)
-        layer.forward(dQ, dK, dV, out=O)
-        hO.copy_(O, non_blocking=True)
+        if shard_mode:
+            dQ.copy_(hQ, non_blocking=True); dK.copy_(hK, non_blocking=True); dV.copy_(hV, non_blocking=True)
+            layer.forward(dQ, dK, dV, out=O)
+            hO.copy_(O, non_blocking=True)
+        else:
+            # the layer's host-buffer entry: K and V first, Q in groups of frames under the attention of the group before
+            layer.forward_host(hQ, hK, hV, hO)
 
     e2e_step()
     barrier()

@@ -63,10 +63,73 @@ class SubsampledGlobalAttention:
 
     __call__ = forward
 
+    def forward_host(self, hQ, hK, hV, hO, n_chunks=8):
+        """The layer on host buffers (pinned memory), with the copies hidden behind the kernels.
+
+        K and V go to the device first (the compaction and the mean need all of them); Q then arrives in
+        ``n_chunks`` groups of frames on a copy stream while the attention of the previous group runs
+        (``avggt_global_attn_shard``: the queries of a frame range against the whole sequence's compact keys), and
+        every group's output leaves on a second copy stream.  Everything is ordered with events; on return the
+        current stream waits for the last output copy.  The device staging buffers are allocated on first use.
+        """
+        p = self.params
+        dev = self.device
+        cur = torch.cuda.current_stream(dev)
+        if not hasattr(self, "_host_path"):
+            shape = (self.n_tok, p.n_heads, p.head_dim)
+            self._host_path = dict(
+                Q=torch.empty(shape, dtype=torch.bfloat16, device=dev), K=torch.empty(shape, dtype=torch.bfloat16, device=dev),
+                V=torch.empty(shape, dtype=torch.bfloat16, device=dev), O=torch.empty(shape, dtype=torch.bfloat16, device=dev),
+                h2d=torch.cuda.Stream(dev), d2h=torch.cuda.Stream(dev),
+                # one status block per group of frames, so that no launch clears what an earlier one reported
+                ws=torch.zeros((max(1, p.n_frames), max(self.attn_ws_bytes, 256)), dtype=torch.uint8, device=dev))
+        hp = self._host_path
+        dQ, dK, dV, dO, h2d, d2h = hp["Q"], hp["K"], hp["V"], hp["O"], hp["h2d"], hp["d2h"]
+        L = p.tokens_per_frame
+        n_chunks = max(1, min(n_chunks, p.n_frames))
+        bounds = [round(i * p.n_frames / n_chunks) for i in range(n_chunks + 1)]
+        keep_first = bool(p.flags & B.AVGGT_FLAG_KEEP_FIRST_FRAME)
+        h2d.wait_stream(cur)
+        d2h.wait_stream(cur)
+        with torch.cuda.device(dev):
+            with torch.cuda.stream(h2d):
+                dK.copy_(hK, non_blocking=True)
+                dV.copy_(hV, non_blocking=True)
+                kv_ready = torch.cuda.Event()
+                kv_ready.record(h2d)
+                q_ready = []
+                for c in range(n_chunks):
+                    sl = slice(bounds[c] * L, bounds[c + 1] * L)
+                    dQ[sl].copy_(hQ[sl], non_blocking=True)
+                    ev = torch.cuda.Event()
+                    ev.record(h2d)
+                    q_ready.append(ev)
+            cur.wait_event(kv_ready)
+            self.build_kv(dK, dV)
+            for c in range(n_chunks):
+                f0, f1 = bounds[c], bounds[c + 1]
+                sl = slice(f0 * L, f1 * L)
+                cp = B.make_params(f1 - f0, p.grid_h, p.grid_w, p.n_special, p.n_heads, p.head_dim, p.sigma, diag=p.diag,
+                                   mean_fill=p.mean_fill, softmax_scale=p.softmax_scale,
+                                   keep_first_frame=keep_first and f0 == 0)
+                cur.wait_event(q_ready[c])
+                B.avggt_global_attn_shard(cp, self.M, self.n_dropped, dQ[sl], dK[sl], dV[sl], self.Kc, self.Vc, self.kmean,
+                                          self.vmean, dO[sl], None, hp["ws"][c], hp["ws"][c].numel(), cur.cuda_stream)
+                done = torch.cuda.Event()
+                done.record(cur)
+                d2h.wait_event(done)
+                with torch.cuda.stream(d2h):
+                    hO[sl].copy_(dO[sl], non_blocking=True)
+            cur.wait_stream(d2h)
+        return hO
+
     def check_status(self):
         """Synchronises the device and raises if a device-side wait gave up."""
         torch.cuda.synchronize(self.device)
         B.avggt_check_status(self.attn_ws)
+        if hasattr(self, "_host_path"):
+            for ws in self._host_path["ws"]:
+                B.avggt_check_status(ws)
 
     def _check_inputs(self, *tensors):
         shape = (self.n_tok, self.params.n_heads, self.params.head_dim)

@@ -287,3 +287,23 @@ def test_extreme_values_stay_finite():
     assert torch.isfinite(O.float()).all() and torch.isfinite(layer.lse).all()
     Kh, Vh = _host(K), _host(V)
     _check_attn(ocfg, Q, Kh, Vh, O, lse=None)
+
+
+def test_host_buffer_forward_matches_the_device_forward():
+    """forward_host (K/V first, Q in groups of frames on a copy stream, outputs leaving on another) gives the very
+    bits of forward on resident tensors, for a frame count that does not divide into the groups, with and without
+    the uncompressed first frame."""
+    for kff in (0, 1):
+        wl = inputs.Workload("host", 11, 12, 13, 5, 4, 64, 4, 1, 2, "proj", keep_first_frame=kff)
+        params, ocfg = _cfgs(wl)
+        Q, K, V = inputs.make_qkv(wl, seed=21, device="cuda")
+        layer = P.SubsampledGlobalAttention(params)
+        O = layer.forward(Q, K, V).clone()
+        layer.check_status()
+        hQ, hK, hV = (t.cpu().pin_memory() for t in (Q, K, V))
+        hO = torch.full_like(hQ, float("nan")).pin_memory()
+        for n_chunks in (1, 4, 50):
+            hO.fill_(float("nan"))
+            layer.forward_host(hQ, hK, hV, hO, n_chunks=n_chunks)
+            layer.check_status()
+            assert torch.equal(hO, O.cpu()), n_chunks
