@@ -1,31 +1,36 @@
 // Subsampled global attention (Sec. 4.3 of the AVGGT paper) as one fused,
-// warp-specialised flash-style kernel for sm_100a.
+// warp-specialised flash-style kernel for sm_100a; the same kernel runs frame
+// attention (Sec. 4.2) as many small dense problems.
 //
-// One CTA owns two tiles of 128 query rows of one head.  Roles (20 warps):
-//   warps 0-15  softmax.  Warpgroup g = 2 t + h works on query tile t and on
-//               columns [64 h, 64 h + 64) of every 128-key step; within it, warp q
-//               owns rows [32 q, 32 q + 32) (the tensor-memory lanes a warp may
-//               touch), one row per thread.  The two threads that share a row
-//               exchange their half-row maxima through shared memory every step
-//               and their partial sums once at the end.  Four softmax warps per
-//               scheduler keep the exponential unit busy while others wait on
-//               tensor memory, barriers or instruction fetch.
-//   warp  16    TMA producer: Q tiles once, then the compacted K/V of the head
-//               through a ring of shared-memory stages (128-byte swizzle); the
-//               last two ring items are the K/V rows of the CTA's own queries
-//               (the preserved diagonal)
+// A work item is two tiles of 128 query rows of one head.  In the subsampled
+// layer a CTA has one work item (hundreds of key steps); in frame attention one
+// CTA per SM walks over many (a dozen key steps each), so that the next item's
+// loads and first product run under the current item's epilogue.
+// Roles (20 warps):
+//   warps 0-15  softmax.  Warp 8 t + 4 h + q works on query tile t, rows
+//               [32 q + 16 h, 32 q + 16 h + 16), all 128 columns of a key step.
+//               It reads tensor memory in the 16-lane shapes, which spread a row
+//               over the four threads of a quad (two rows per thread): a row's
+//               maximum and sums are two shuffles away and every row lives in one
+//               warp.  Four softmax warps per scheduler keep the exponential unit
+//               busy while others wait on tensor memory or barriers.
+//   warp  16    TMA producer: Q tiles once per work item, then the compacted K/V
+//               of the head through a ring of shared-memory stages (128-byte
+//               swizzle); in the subsampled layer the last two ring items are the
+//               K/V rows of the CTA's own queries (the preserved diagonal)
 //   warps 17-18 MMA issuers, one per query tile: S_t = Q_t Kc_j^T and
 //               O_t += P_t Vc_j with tcgen05.mma, bf16 operands, fp32
 //               accumulators in tensor memory
 //   warp  19    idle (it completes the fifth warpgroup so that registers can
 //               be moved to the softmax warpgroups)
 // Tensor memory per tile: S 128 columns (fp32), P 64 columns (bf16 pairs),
-// O 64 columns (fp32); 512 columns in all.  A softmax thread pulls its half row
-// of S into registers and frees S at once, so the next Q K^T runs under the
-// exponentials; P V of step j runs under the softmax of step j+1.  The
-// accumulator is rescaled lazily: only when the running maximum grew by more
-// than 2^8 since the last rescale.  The epilogue folds the diagonal and the
-// mean-fill column into the same normalisation:
+// O 64 columns (fp32); 512 columns in all.  A softmax thread pulls its 64 scores
+// of S into registers and the warp frees its rows at once, so the next Q K^T runs
+// under the exponentials; P V of step j runs under the softmax of step j+1.  The
+// two tiles take turns in the exponential phase.  The accumulator is rescaled
+// lazily: only when the running maximum grew by more than 2^8 since the last
+// rescale.  The epilogue folds the diagonal and the mean-fill column into the
+// same normalisation:
 //   O = (a_S O_S + p_d v_i + p_m vmean) / (a_S l_S + p_d + p_m).
 #include <mutex>
 
@@ -69,6 +74,11 @@ constexpr float kRescaleThreshold = 8.0f;   // log2 units
 #ifndef AVGGT_PINGPONG
 #define AVGGT_PINGPONG 1
 #endif
+// The turn is handed to the other tile after this group of 32 keys (0..3) of a step; 3 = at the end.  Handing over
+// early lets the other tile's warps wake up and start while this tile still feeds the exponential unit.
+#ifndef AVGGT_HANDOVER_GROUP
+#define AVGGT_HANDOVER_GROUP 1
+#endif
 constexpr int kPolyEighths = AVGGT_POLY_EIGHTHS;
 
 struct AttnArgs {
@@ -102,7 +112,6 @@ struct __align__(8) Barriers {
   uint64_t p_full[kQTiles];    // softmax -> MMA: P_t(j) stored (and O_t rescaled)
   uint64_t o_done[kQTiles];    // MMA -> softmax: P_t(j) V_j has completed
   uint64_t turn[kQTiles][4];   // both warps of rows [32 q, 32 q + 32) of the other tile -> this tile's: the exponential unit is yours
-  uint64_t pair[kQTiles][4];   // the two warps that share rows [32 q, 32 q + 32) of tile t: my half-row value is in shared memory
   uint64_t mma_idle[kQTiles];  // MMA issuer t -> itself: every tcgen05.mma it issued has completed
   uint32_t tmem_base;
   uint32_t abort_flag;
@@ -417,85 +426,147 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1
 template <int kPoly>
 __device__ __forceinline__ constexpr bool pair_uses_poly(int g) { return ((g + 1) * kPoly) / 8 != (g * kPoly) / 8; }
 
-// Values the two threads of a row hand to each other through shared memory.
-struct PairExchange {
-  float step[kQTiles][2][2][kTileQ];    // [tile][step parity][half][row]: half-row maximum of a step
-  float final[kQTiles][2][2][kTileQ];   // [tile][which sum][half][row]: partial sums, once, in the epilogue
-};
-
-// 64 scores of one query row (a half row) -> bf16 probabilities, stored to tensor memory at tP,
-// relative to the reference maximum folded into neg_m2; adds to the sums for the normaliser (of
-// the rounded values) and for the log-sum-exp (unrounded).  Written pair by pair in dependency
-// order; the instruction scheduler interleaves the pairs.
-template <bool kLse, int kPoly>
-__device__ __forceinline__ void softmax_half_row(const uint32_t (&s)[64], uint64_t scale2, uint64_t neg_m2, float& sum_lo,
-                                                 float& sum_hi, uint64_t& sum_exact2, uint32_t tP) {
-#pragma unroll
-  for (int g = 0; g < 4; ++g) {
-    uint32_t pk[8];   // P of 16 columns as bf16 pairs
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int c = 16 * g + 2 * i;
-      const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), scale2, neg_m2);
-      float p0, p1;
-      if (pair_uses_poly<kPoly>(i)) {
-        exp2_poly_pair(x2, p0, p1);
-      } else {
-        float x0, x1;
-        unpack_f32x2(x2, x0, x1);
-        p0 = ex2_approx(x0);
-        p1 = ex2_approx(x1);
-      }
-      const uint32_t w = pack_bf16x2(p0, p1);
-      pk[i] = w;
-      if (kLse) sum_exact2 = add_f32x2(sum_exact2, pack_f32x2(p0, p1));
-      add_bf16x2_to_f32(w, sum_lo, sum_hi);
-    }
-    tmem_st8(tP + g * 8, pk);
-  }
-}
-
-// What a softmax thread knows about itself.
+// What a softmax thread knows about itself.  A softmax warp works on 16 query rows of its tile, all 128 columns
+// of a key step: the tensor-memory lanes [32 q + 16 h, 32 q + 16 h + 16) of the tile.  Its tensor-memory
+// accesses use the 16-lane shapes, which spread a row over the four threads of a quad: thread `lane` holds,
+// of every block of 8 columns, columns 2 i and 2 i + 1 (i = lane % 4) of the rows lane / 4 and lane / 4 + 8.
+// A row's maximum and sums therefore take two shuffles within the quad and no shared memory, and every row
+// is handled inside one warp.
 struct SoftmaxThread {
   int t;        // query tile of the CTA
-  int h;        // which half of the 128 columns of a step (and of the 64 output dimensions)
-  int q;        // warp within the warpgroup: rows [32 q, 32 q + 32)
-  int r;        // row within the tile
+  int h;        // which 16 of the 32 lanes of the warp's tensor-memory quarter
+  int q;        // tensor-memory quarter (and scheduler): lanes [32 q, 32 q + 32)
   int lane;
-  uint32_t tS, tP, tO;   // tensor-memory addresses of its half of S, P and O (lane included)
+  int i;        // position in the quad: columns 2 i, 2 i + 1 of every 8
+  int r[2];     // the thread's two rows within the tile
+  uint32_t tS, tP, tO;   // tensor-memory addresses (first lane of the warp's 16) of S, P and O of the tile
 };
 
-// Meeting point of the two warps that share the rows of `me`: returns once both have arrived for
-// the given phase (one phase per step, one more in the epilogue).  What either wrote to shared
-// memory before arriving is visible to the other afterwards.
-__device__ __forceinline__ bool pair_sync(uint32_t phase, const SoftmaxThread& me, Barriers* bars, const AttnArgs& a) {
-  __syncwarp();
-  if (me.lane == 0) mbar_arrive(smem_u32(&bars->pair[me.t][me.q]));
-  return wait_bar(&bars->pair[me.t][me.q], phase & 1, bars, a, 60 + me.t, phase);
+// tensor memory <-> registers in the 16-lane shapes (layout above): S (128 columns) and O (64 columns) as 32-bit
+// columns, P as 64 columns of bf16 pairs
+__device__ __forceinline__ void tmem_ld_rows16_c128(uint32_t taddr, uint32_t (&r)[64]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
+      "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "
+      "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]),
+        "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]),
+        "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]),
+        "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]),
+        "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_rows16_c64(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_rows16_c64(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.16x256b.x8.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+// bf16 pairs of 4 blocks of 8 keys: register 2 n + hi -> row hi of the thread, pair column 4 n + i
+__device__ __forceinline__ void tmem_st_rows16_p16(uint32_t taddr, const uint32_t (&r)[8]) {
+  asm volatile("tcgen05.st.sync.aligned.16x128b.x4.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
 }
 
-// One step of the online softmax of half a query row: S_t(j) in tensor memory -> P_t(j) in
-// tensor memory, running reference maximum and partial sums updated.
+// value over the four threads of a quad
+__device__ __forceinline__ float quad_max(float v) {
+  v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 1));
+  return fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 2));
+}
+__device__ __forceinline__ float quad_sum(float v) {
+  v += __shfl_xor_sync(0xffffffffu, v, 1);
+  return v + __shfl_xor_sync(0xffffffffu, v, 2);
+}
+
+// Running state of the thread's two rows (the same in all four threads of a quad, except the partial sums).
+struct RowState {
+  float m_used[2];    // reference maximum of the stored exponentials (log2 units)
+  float l_run[2];     // this thread's part of the sum of the bf16-rounded 2^(scale_log2 * s - m_used): normaliser of O
+  float l_exact[2];   // the same sum without the rounding: log-sum-exp output only
+};
+
+// The thread's 64 scores of a key step (register 4 b + 2 hi + e: row hi, column 8 b + 2 i + e) -> bf16
+// probabilities, stored to tensor memory at tP, relative to the rows' reference maxima folded into neg_m2; adds
+// to the sums for the normaliser (of the rounded values) and for the log-sum-exp (unrounded).  Written pair by
+// pair in dependency order; the instruction scheduler interleaves the pairs.
+template <bool kLse, int kPoly>
+__device__ __forceinline__ void softmax_rows(const uint32_t (&s)[64], uint64_t scale2, const uint64_t (&neg_m2)[2],
+                                             float (&sum_lo)[2], float (&sum_hi)[2], uint64_t (&sum_exact2)[2], uint32_t tP,
+                                             uint32_t turn_bar, int lane) {
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    uint32_t pk[8];   // P of 32 keys x 2 rows as bf16 pairs
+#pragma unroll
+    for (int n = 0; n < 4; ++n) {
+#pragma unroll
+      for (int hi = 0; hi < 2; ++hi) {
+        const int c = 4 * (4 * g + n) + 2 * hi;
+        const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), scale2, neg_m2[hi]);
+        float p0, p1;
+        if (pair_uses_poly<kPoly>(2 * n + hi)) {
+          exp2_poly_pair(x2, p0, p1);
+        } else {
+          float x0, x1;
+          unpack_f32x2(x2, x0, x1);
+          p0 = ex2_approx(x0);
+          p1 = ex2_approx(x1);
+        }
+        const uint32_t w = pack_bf16x2(p0, p1);
+        pk[2 * n + hi] = w;
+        if (kLse) sum_exact2[hi] = add_f32x2(sum_exact2[hi], pack_f32x2(p0, p1));
+        add_bf16x2_to_f32(w, sum_lo[hi], sum_hi[hi]);
+      }
+    }
+    tmem_st_rows16_p16(tP + g * 16, pk);
+#if AVGGT_PINGPONG
+    // the store above is ordered before the arrival, and with it this group's exponentials
+    if (g == AVGGT_HANDOVER_GROUP) {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(turn_bar);
+    }
+#endif
+  }
+}
+
+// One step of the online softmax of the thread's two rows: S_t(j) in tensor memory -> P_t(j) in tensor
+// memory, running reference maxima and partial sums updated.
 //
-// The half row's 64 scores are pulled into registers at once and the thread's share of S_t is
-// released, so that the next Q K^T runs under this step's exponentials.  The row maximum (of both
-// halves, exchanged with the partner thread) decides whether the reference maximum moves (lazy
-// rescale); both threads of a row take the same decision from the same numbers.
-// j: step within the work item; g: the tile's steps in the CTA's earlier work items; pair_phase: meetings with
-// the partner thread so far.  kPoly: pairs per eight whose exponential is a polynomial.  kLse: also keep the sum of the
-// unrounded exponentials, for the log-sum-exp output.  kMasked: columns >= valid are excluded
-// (valid counts from this thread's first column and may be <= 0).
+// The 64 scores are pulled into registers at once and the warp's share of S_t is released, so that the next
+// Q K^T runs under this step's exponentials.  The row maxima (two shuffles within the quad) decide whether a
+// reference maximum moves (lazy rescale).
+// j: step within the work item; g: the tile's steps in the CTA's earlier work items.  kPoly: pairs per eight
+// whose exponential is a polynomial.  kLse: also keep the sum of the unrounded exponentials, for the
+// log-sum-exp output.  kMasked: columns >= valid are excluded (valid may be <= 0).
 template <bool kMasked, bool kLse, int kPoly>
-__device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int g, uint32_t pair_phase, int valid,
-                                             float scale_log2, float& m_used, float& l_run, float& l_exact, Barriers* bars,
-                                             PairExchange* px, const AttnArgs& a) {
+__device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int g, int valid, float scale_log2,
+                                             RowState& st, Barriers* bars, const AttnArgs& a) {
   const int gj = g + j;   // this tile's key steps so far, over all work items of the CTA: the phase of the per-step barriers
   uint32_t s[64];
-  {
-    uint32_t (&s2)[2][32] = reinterpret_cast<uint32_t (&)[2][32]>(s);
-    tmem_ld32(me.tS, s2[0]);
-    tmem_ld32(me.tS + 32, s2[1]);
-  }
+  tmem_ld_rows16_c128(me.tS, s);
   tmem_wait_ld();
   tc_fence_before();
   __syncwarp();
@@ -503,45 +574,42 @@ __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int
 
   if (kMasked) {
 #pragma unroll
-    for (int i = 0; i < 64; ++i)
-      if (i >= valid) s[i] = __float_as_uint(-INFINITY);
+    for (int c = 0; c < 64; ++c)
+      if (8 * (c >> 2) + 2 * me.i + (c & 1) >= valid) s[c] = __float_as_uint(-INFINITY);
   }
-  float mx[2];
+  float alpha[2];
+  bool jump_any = false;
 #pragma unroll
-  for (int c = 0; c < 2; ++c) {
-    mx[c] = fmaxf(__uint_as_float(s[32 * c]), __uint_as_float(s[32 * c + 1]));
+  for (int hi = 0; hi < 2; ++hi) {
+    float mx = fmaxf(__uint_as_float(s[2 * hi]), __uint_as_float(s[2 * hi + 1]));
 #pragma unroll
-    for (int i = 2; i < 32; i += 2) mx[c] = max3(mx[c], __uint_as_float(s[32 * c + i]), __uint_as_float(s[32 * c + i + 1]));
+    for (int b = 1; b < 16; ++b) mx = max3(mx, __uint_as_float(s[4 * b + 2 * hi]), __uint_as_float(s[4 * b + 2 * hi + 1]));
+    const float tile_max = quad_max(mx) * scale_log2;
+    // lazy rescale: keep the old reference maximum unless the new one is far above it
+    const bool jump = tile_max > st.m_used[hi] + kRescaleThreshold;
+    alpha[hi] = 1.0f;
+    if (jump) {
+      alpha[hi] = ex2_approx(st.m_used[hi] - tile_max);   // 0 on the first tile (m_used = -inf)
+      st.m_used[hi] = tile_max;
+      st.l_run[hi] *= alpha[hi];
+      if (kLse) st.l_exact[hi] *= alpha[hi];
+    }
+    jump_any = jump_any || jump;
   }
-  const float half_max = fmaxf(mx[0], mx[1]);
-  // two slots, by step parity: the partner may still be reading the previous step's value
-  px->step[me.t][gj & 1][me.h][me.r] = half_max;
-  if (!pair_sync(pair_phase, me, bars, a)) return false;
-  const float other_max = *reinterpret_cast<const volatile float*>(&px->step[me.t][gj & 1][me.h ^ 1][me.r]);
-  const float tile_max = fmaxf(half_max, other_max) * scale_log2;
-  // lazy rescale: keep the old reference maximum unless the new one is far above it
-  const bool jump = tile_max > m_used + kRescaleThreshold;
-  float alpha = 1.0f;
-  if (jump) {
-    alpha = ex2_approx(m_used - tile_max);   // 0 on the first tile (m_used = -inf)
-    m_used = tile_max;
-    l_run *= alpha;
-    if (kLse) l_exact *= alpha;
-  }
-  const bool rescale = (j > 0) && __any_sync(0xffffffffu, jump);
+  const bool rescale = (j > 0) && __any_sync(0xffffffffu, jump_any);
 
   // P_t(j-1) must have been consumed, and O_t be at rest, before either is written
   if (j > 0) {
     if (!wait_bar(&bars->o_done[me.t], (gj - 1) & 1, bars, a, 30 + me.t, gj)) return false;
     tc_fence_after();
   }
-  if (rescale) {   // this thread's 32 of the row's 64 accumulator columns
+  if (rescale) {   // the warp's 16 rows of the accumulator: register 4 b + 2 hi + e is row hi
     uint32_t o[32];
-    tmem_ld32(me.tO, o);
+    tmem_ld_rows16_c64(me.tO, o);
     tmem_wait_ld();
 #pragma unroll
-    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-    tmem_st32(me.tO, o);
+    for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha[(c >> 1) & 1]);
+    tmem_st_rows16_c64(me.tO, o);
   }
 #if AVGGT_PINGPONG
   // this tile's turn on the exponential unit: the other tile's two warps on this scheduler have left their phase
@@ -551,20 +619,19 @@ __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int
   // exponentials, rounded to bf16 for the value product; the normaliser sums the
   // rounded values so that numerator and denominator carry the same weights
   const uint64_t scale2 = pack_f32x2(scale_log2, scale_log2);
-  const uint64_t neg_m2 = pack_f32x2(-m_used, -m_used);
-  float sum_lo = 0.f, sum_hi = 0.f;   // even and odd columns
-  uint64_t sum_exact2 = pack_f32x2(0.f, 0.f);
-  softmax_half_row<kLse, kPoly>(s, scale2, neg_m2, sum_lo, sum_hi, sum_exact2, me.tP);
-#if AVGGT_PINGPONG
-  __syncwarp();
-  if (me.lane == 0) mbar_arrive(smem_u32(&bars->turn[me.t ^ 1][me.q]));
-#endif
-
-  l_run += sum_lo + sum_hi;
-  if (kLse) {
-    float sum_a, sum_b;
-    unpack_f32x2(sum_exact2, sum_a, sum_b);
-    l_exact += sum_a + sum_b;
+  const uint64_t neg_m2[2] = {pack_f32x2(-st.m_used[0], -st.m_used[0]), pack_f32x2(-st.m_used[1], -st.m_used[1])};
+  float sum_lo[2] = {0.f, 0.f}, sum_hi[2] = {0.f, 0.f};   // even and odd columns
+  uint64_t sum_exact2[2] = {pack_f32x2(0.f, 0.f), pack_f32x2(0.f, 0.f)};
+  softmax_rows<kLse, kPoly>(s, scale2, neg_m2, sum_lo, sum_hi, sum_exact2, me.tP,
+                            smem_u32(&bars->turn[me.t ^ 1][me.q]), me.lane);
+#pragma unroll
+  for (int hi = 0; hi < 2; ++hi) {
+    st.l_run[hi] += sum_lo[hi] + sum_hi[hi];
+    if (kLse) {
+      float sum_a, sum_b;
+      unpack_f32x2(sum_exact2[hi], sum_a, sum_b);
+      st.l_exact[hi] += sum_a + sum_b;
+    }
   }
   tmem_wait_st();
   tc_fence_before();
@@ -573,50 +640,38 @@ __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int
   return true;
 }
 
+// 4-byte word (two bf16) number w (0..31) of row r of a 128-byte-swizzled tile
+__device__ __forceinline__ uint32_t ld_swizzled_word(const uint8_t* tile, int r, int w) {
+  return *reinterpret_cast<const uint32_t*>(tile + r * 128 + (((w >> 2) ^ (r & 7)) << 4) + ((w & 3) << 2));
+}
+
 // One work item of a softmax thread: the key steps, then the epilogue.  g: this tile's key steps in the CTA's earlier
-// work items; pair_phase: meetings with the partner thread so far; n_done: work items before this one.
-__device__ __forceinline__ bool softmax_item(const AttnArgs& a, Barriers* bars, PairExchange* px, const SmemLayout& sm,
-                                             const SoftmaxThread& me, const CtaProblem& cta, int g, uint32_t pair_phase,
-                                             int n_done) {
+// work items; n_done: work items before this one.
+__device__ __forceinline__ bool softmax_item(const AttnArgs& a, Barriers* bars, const SmemLayout& sm, const SoftmaxThread& me,
+                                             const CtaProblem& cta, int g, int n_done) {
   const Plan& pl = a.pl;
   const int n_kv = a.n_kv_tiles;
-  const int t = me.t, r = me.r, lane = me.lane;
-  float m_used = -INFINITY;   // reference maximum of the stored exponentials (log2 units); the same in both threads of a row
-  float l_run = 0.f;          // this half's sum of the bf16-rounded 2^(scale_log2 * s - m_used): normaliser of O
-  float l_exact = 0.f;        // the same sum without the rounding: log-sum-exp output only
+  const int t = me.t, lane = me.lane;
+  RowState st;
+#pragma unroll
+  for (int hi = 0; hi < 2; ++hi) { st.m_used[hi] = -INFINITY; st.l_run[hi] = 0.f; st.l_exact[hi] = 0.f; }
   const bool want_lse = a.lse != nullptr;
+
 #pragma unroll 1
   for (int j = 0; j < n_kv; ++j) {
     if (!wait_bar(&bars->s_full[t], (g + j) & 1, bars, a, 40 + t, g + j)) return false;
     tc_fence_after();
-    const int valid_tile = static_cast<int>(a.n_keys - static_cast<int64_t>(j) * kTileKV);
-    const int valid = valid_tile - 64 * me.h;
+    const int valid = static_cast<int>(a.n_keys - static_cast<int64_t>(j) * kTileKV);
     bool ok;
     // the masked (last, ragged) tile keeps every exponential on the special-function unit, where -inf gives an exact 0
-    if (valid_tile < kTileKV) ok = softmax_step<true, true, 0>(me, j, g, pair_phase + j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a);
-    else if (want_lse) ok = softmax_step<false, true, kPolyEighths>(me, j, g, pair_phase + j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a);
-    else ok = softmax_step<false, false, kPolyEighths>(me, j, g, pair_phase + j, valid, a.scale_log2, m_used, l_run, l_exact, bars, px, a);
+    if (valid < kTileKV) ok = softmax_step<true, true, 0>(me, j, g, valid, a.scale_log2, st, bars, a);
+    else if (want_lse) ok = softmax_step<false, true, kPolyEighths>(me, j, g, valid, a.scale_log2, st, bars, a);
+    else ok = softmax_step<false, false, kPolyEighths>(me, j, g, valid, a.scale_log2, st, bars, a);
     if (!ok) return false;
   }
 
-  // ---- epilogue: diagonal and mean-fill terms, normalisation, store of this thread's 32 output dimensions
+  // ---- epilogue: diagonal and mean-fill terms, normalisation, store of this thread's 16 output dimensions of two rows
   const int head = cta.head;
-  const int row = cta.q0 + t * kTileQ + r;           // query token
-  const bool row_valid = row < cta.row_end;
-  bool is_dropped = false;
-  if (row_valid && pl.n_dropped > 0) {
-    const int32_t f = row / pl.L;
-    is_dropped = (a.slot_of_token != nullptr ? a.slot_of_token[row] : compact_slot(pl, f, row - f * pl.L)) < 0;
-  }
-  // the row's sums: mine plus the partner's
-  px->final[t][0][me.h][r] = l_run;
-  px->final[t][1][me.h][r] = l_exact;
-  if (!pair_sync(pair_phase + n_kv, me, bars, a)) return false;
-  const float other_run = *reinterpret_cast<const volatile float*>(&px->final[t][0][me.h ^ 1][r]);
-  const float other_exact = *reinterpret_cast<const volatile float*>(&px->final[t][1][me.h ^ 1][r]);
-  l_run += other_run;
-  l_exact += other_exact;
-
   if (n_kv > 0) {
     if (!wait_bar(&bars->o_done[t], (g + n_kv - 1) & 1, bars, a, 50 + t, g + n_kv)) return false;
     tc_fence_after();
@@ -633,46 +688,10 @@ __device__ __forceinline__ bool softmax_item(const AttnArgs& a, Barriers* bars, 
     if (!wait_bar(&bars->v_full[item % kStages], par, bars, a, 54, item)) return false;
   }
   const uint8_t* sQ = sm.q[t];
-  // base-2 logits of the two extra columns; both threads of a row compute them in full, from the same numbers
-  float l_d = -INFINITY, l_m = -INFINITY;
-  if (a.use_diag && is_dropped) {
-    float acc = 0.f;
-#pragma unroll
-    for (int c = 0; c < 8; ++c) acc = dot_bf16x8(ld_swizzled(sQ, r, c), ld_swizzled(sKd, r, c), acc);
-    l_d = acc * a.scale_log2;
-  }
-  const int64_t count = pl.n_dropped - ((a.use_diag && is_dropped) ? 1 : 0);
-  const bool has_mean = a.use_mean && count > 0;
-  if (has_mean) {
-    const float4* km = reinterpret_cast<const float4*>(a.kmean + head * kHeadDim);
-    float acc = 0.f;
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      const uint4 q = ld_swizzled(sQ, r, c);
-      const float4 k0 = __ldg(km + 2 * c), k1 = __ldg(km + 2 * c + 1);
-      acc = fmaf(__uint_as_float(q.x << 16), k0.x, acc);
-      acc = fmaf(__uint_as_float(q.x & 0xffff0000u), k0.y, acc);
-      acc = fmaf(__uint_as_float(q.y << 16), k0.z, acc);
-      acc = fmaf(__uint_as_float(q.y & 0xffff0000u), k0.w, acc);
-      acc = fmaf(__uint_as_float(q.z << 16), k1.x, acc);
-      acc = fmaf(__uint_as_float(q.z & 0xffff0000u), k1.y, acc);
-      acc = fmaf(__uint_as_float(q.w << 16), k1.z, acc);
-      acc = fmaf(__uint_as_float(q.w & 0xffff0000u), k1.w, acc);
-    }
-    l_m = acc * a.scale_log2;
-    if (pl.mean_fill == AVGGT_MEAN_FILL) l_m += log2f(static_cast<float>(count));
-  }
-  const float m_fin = fmaxf(m_used, fmaxf(l_d, l_m));
-  const float a_s = exp2f(m_used - m_fin);
-  const float p_d = exp2f(l_d - m_fin);              // 0 when the term is absent
-  const float p_m = exp2f(l_m - m_fin);
-  const float z = fmaf(l_run, a_s, p_d + p_m);
-  const float inv_z = 1.0f / z;
-  const float w_s = a_s * inv_z, w_d = p_d * inv_z, w_m = p_m * inv_z;
 
-  uint32_t o[32];
+  uint32_t o[32];   // register 4 b + 2 hi + e: row hi, output dimension 8 b + 2 i + e
   if (n_kv > 0) {
-    tmem_ld32(me.tO, o);
+    tmem_ld_rows16_c64(me.tO, o);
     tmem_wait_ld();
     // O_t is in registers: the next work item's first P V may overwrite it
     tc_fence_before();
@@ -680,69 +699,111 @@ __device__ __forceinline__ bool softmax_item(const AttnArgs& a, Barriers* bars, 
     if (lane == 0) mbar_arrive(smem_u32(&bars->o_free[t]));
   } else {   // no retained keys at all: the accumulator was never written
 #pragma unroll
-    for (int i = 0; i < 32; ++i) o[i] = 0u;
+    for (int c = 0; c < 32; ++c) o[c] = 0u;
   }
-  if (row_valid) {
-    uint4* dst = reinterpret_cast<uint4*>(a.O + (static_cast<size_t>(row) * pl.H + head) * kHeadDim) + 4 * me.h;
-    const float4* vm = reinterpret_cast<const float4*>(a.vmean + head * kHeadDim) + 8 * me.h;
+
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      float v[8];
+  for (int hi = 0; hi < 2; ++hi) {
+    const int r = me.r[hi];
+    const int row = cta.q0 + t * kTileQ + r;           // query token
+    const bool row_valid = row < cta.row_end;
+    bool is_dropped = false;
+    if (row_valid && pl.n_dropped > 0) {
+      const int32_t f = row / pl.L;
+      is_dropped = (a.slot_of_token != nullptr ? a.slot_of_token[row] : compact_slot(pl, f, row - f * pl.L)) < 0;
+    }
+    // the row's sums over its four threads
+    const float l_run = quad_sum(st.l_run[hi]);
+    const float l_exact = quad_sum(st.l_exact[hi]);
+    const float m_used = st.m_used[hi];
+    // base-2 logits of the two extra columns: each thread of the quad takes its 16 dimensions, then the quad adds up
+    // (every thread runs the shuffles; rows without the term carry zeros)
+    const bool has_diag = a.use_diag && is_dropped;
+    const int64_t count = pl.n_dropped - (has_diag ? 1 : 0);
+    const bool has_mean = a.use_mean && count > 0;
+    float acc_d = 0.f, acc_m = 0.f;
+    if (a.use_diag || a.use_mean) {
 #pragma unroll
-      for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(o[c * 8 + e]) * w_s;
-      if (w_d != 0.f) {
-        const uint4 vd = ld_swizzled(sVd, r, 4 * me.h + c);
-        const uint32_t w[4] = {vd.x, vd.y, vd.z, vd.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          v[2 * e] = fmaf(w_d, __uint_as_float(w[e] << 16), v[2 * e]);
-          v[2 * e + 1] = fmaf(w_d, __uint_as_float(w[e] & 0xffff0000u), v[2 * e + 1]);
+      for (int b = 0; b < 8; ++b) {
+        const uint32_t qw = ld_swizzled_word(sQ, r, 4 * b + me.i);
+        const float q0 = __uint_as_float(qw << 16), q1 = __uint_as_float(qw & 0xffff0000u);
+        if (has_diag) {
+          const uint32_t kw = ld_swizzled_word(sKd, r, 4 * b + me.i);
+          acc_d = fmaf(q0, __uint_as_float(kw << 16), acc_d);
+          acc_d = fmaf(q1, __uint_as_float(kw & 0xffff0000u), acc_d);
+        }
+        if (has_mean) {
+          const float2 km = __ldg(reinterpret_cast<const float2*>(a.kmean + head * kHeadDim + 8 * b + 2 * me.i));
+          acc_m = fmaf(q0, km.x, acc_m);
+          acc_m = fmaf(q1, km.y, acc_m);
         }
       }
-      if (has_mean) {
-        const float4 m0 = __ldg(vm + 2 * c), m1 = __ldg(vm + 2 * c + 1);
-        v[0] = fmaf(w_m, m0.x, v[0]); v[1] = fmaf(w_m, m0.y, v[1]); v[2] = fmaf(w_m, m0.z, v[2]); v[3] = fmaf(w_m, m0.w, v[3]);
-        v[4] = fmaf(w_m, m1.x, v[4]); v[5] = fmaf(w_m, m1.y, v[5]); v[6] = fmaf(w_m, m1.z, v[6]); v[7] = fmaf(w_m, m1.w, v[7]);
-      }
-      uint4 out;
-      out.x = pack_bf16x2(v[0], v[1]);
-      out.y = pack_bf16x2(v[2], v[3]);
-      out.z = pack_bf16x2(v[4], v[5]);
-      out.w = pack_bf16x2(v[6], v[7]);
-      dst[c] = out;
+      acc_d = quad_sum(acc_d);
+      acc_m = quad_sum(acc_m);
     }
-    if (want_lse && me.h == 0) {
-      const float z_exact = fmaf(l_exact, a_s, p_d + p_m);
-      a.lse[static_cast<size_t>(row) * pl.H + head] = (m_fin + log2f(z_exact)) * 0.6931471805599453f;
+    float l_d = -INFINITY, l_m = -INFINITY;
+    if (has_diag) l_d = acc_d * a.scale_log2;
+    if (has_mean) {
+      l_m = acc_m * a.scale_log2;
+      if (pl.mean_fill == AVGGT_MEAN_FILL) l_m += log2f(static_cast<float>(count));
+    }
+    const float m_fin = fmaxf(m_used, fmaxf(l_d, l_m));
+    const float a_s = exp2f(m_used - m_fin);
+    const float p_d = exp2f(l_d - m_fin);              // 0 when the term is absent
+    const float p_m = exp2f(l_m - m_fin);
+    const float z = fmaf(l_run, a_s, p_d + p_m);
+    const float inv_z = 1.0f / z;
+    const float w_s = a_s * inv_z, w_d = p_d * inv_z, w_m = p_m * inv_z;
+    if (row_valid) {
+      uint32_t* dst = reinterpret_cast<uint32_t*>(a.O + (static_cast<size_t>(row) * pl.H + head) * kHeadDim);
+#pragma unroll
+      for (int b = 0; b < 8; ++b) {
+        float v0 = __uint_as_float(o[4 * b + 2 * hi]) * w_s, v1 = __uint_as_float(o[4 * b + 2 * hi + 1]) * w_s;
+        if (w_d != 0.f) {
+          const uint32_t vw = ld_swizzled_word(sVd, r, 4 * b + me.i);
+          v0 = fmaf(w_d, __uint_as_float(vw << 16), v0);
+          v1 = fmaf(w_d, __uint_as_float(vw & 0xffff0000u), v1);
+        }
+        if (has_mean) {
+          const float2 vm = __ldg(reinterpret_cast<const float2*>(a.vmean + head * kHeadDim + 8 * b + 2 * me.i));
+          v0 = fmaf(w_m, vm.x, v0);
+          v1 = fmaf(w_m, vm.y, v1);
+        }
+        dst[4 * b + me.i] = pack_bf16x2(v0, v1);
+      }
+      if (want_lse && me.i == 0) {
+        const float z_exact = fmaf(l_exact, a_s, p_d + p_m);
+        a.lse[static_cast<size_t>(row) * pl.H + head] = (m_fin + log2f(z_exact)) * 0.6931471805599453f;
+      }
     }
   }
   return true;
 }
 
-__device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, PairExchange* px, const SmemLayout& sm,
-                                             uint32_t tmem, int warp, int lane) {
+__device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, const SmemLayout& sm, uint32_t tmem, int warp,
+                                             int lane) {
   SoftmaxThread me;
   me.t = warp >> 3;
   me.h = (warp >> 2) & 1;
   me.q = warp & 3;
   me.lane = lane;
-  me.r = 32 * me.q + lane;
-  const uint32_t tile_base = tmem + me.t * kTmemTileStride + (static_cast<uint32_t>(32 * me.q) << 16);   // TMEM lane = row
-  me.tS = tile_base + 64 * me.h;
-  me.tP = tile_base + kColP + 32 * me.h;
-  me.tO = tile_base + kColO + 32 * me.h;
+  me.i = lane & 3;
+  me.r[0] = 32 * me.q + 16 * me.h + (lane >> 2);
+  me.r[1] = me.r[0] + 8;
+  const uint32_t tile_base = tmem + me.t * kTmemTileStride + (static_cast<uint32_t>(32 * me.q + 16 * me.h) << 16);   // TMEM lane = row
+  me.tS = tile_base;
+  me.tP = tile_base + kColP;
+  me.tO = tile_base + kColO;
 #if AVGGT_PINGPONG
   // tile 0 goes first: tile 1 hands it the first turn
   if (me.t == 1 && lane == 0) mbar_arrive(smem_u32(&bars->turn[0][me.q]));
 #endif
   const int n_kv = a.n_kv_tiles;
   int g = 0, n_done = 0;
-  uint32_t pair_phase = 0;
 #pragma unroll 1
   for (int item = blockIdx.x; item < a.n_work; item += gridDim.x) {
-    if (!softmax_item(a, bars, px, sm, me, work_item(a, item), g, pair_phase, n_done)) return;
+    if (!softmax_item(a, bars, sm, me, work_item(a, item), g, n_done)) return;
     g += n_kv;
-    pair_phase += static_cast<uint32_t>(n_kv) + 1u;   // one meeting per step and one in the epilogue
     ++n_done;
   }
 }
@@ -759,7 +820,6 @@ global_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   sm.k = smem + kQTiles * kTileBytes;
   sm.v = sm.k + kStages * kTileBytes;
   __shared__ Barriers bars;
-  __shared__ PairExchange pair_exchange;
 
   const int tid = threadIdx.x;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // warp-uniform by construction
@@ -780,7 +840,6 @@ global_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       mbar_init(smem_u32(&bars.s_free[t]), kSoftmaxWarps / kQTiles);
       mbar_init(smem_u32(&bars.p_full[t]), kSoftmaxWarps / kQTiles);
       mbar_init(smem_u32(&bars.o_done[t]), 1);
-      for (int w = 0; w < 4; ++w) mbar_init(smem_u32(&bars.pair[t][w]), 2);
       for (int w = 0; w < 4; ++w) mbar_init(smem_u32(&bars.turn[t][w]), 2);
       mbar_init(smem_u32(&bars.mma_idle[t]), 1);
       mbar_init(smem_u32(&bars.o_free[t]), kSoftmaxWarps / kQTiles);
@@ -799,7 +858,7 @@ global_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
   if (warp < kSoftmaxWarps) {
     reg_inc<kRegsSoftmax>();
-    softmax_role(a, &bars, &pair_exchange, sm, tmem, warp, tid & 31);
+    softmax_role(a, &bars, sm, tmem, warp, tid & 31);
   } else {
     reg_dec<kRegsOther>();
     if (warp == kTmaWarp) producer_role(&tm_q, &tm_k, &tm_v, &tm_kc, &tm_vc, a, &bars, sm);
