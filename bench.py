@@ -42,8 +42,8 @@ from paper_2512_02541_b200 import inputs  # noqa: E402
 # profiles/; None where no capture covers the workload.  Both kernels are captured on the 30-frame copy of the
 # headline layer (profiles/*_vggt_n30_s9.md); their traffic is proportional to the frame count, so the 800-frame
 # figures are those captures x 800/30.
-_ATTN_N30_S9 = 0.275029760e9 + 0.067800832e9
-_BUILD_N30_S9 = 0.168853760e9 + 0.007183104e9
+_ATTN_N30_S9 = 0.275695104e9 + 0.067074048e9
+_BUILD_N30_S9 = 0.168855296e9 + 0.009879808e9
 NCU_TRAFFIC = {
     "vggt_n30_s9": {"global_attn_kernel": _ATTN_N30_S9, "build_kv_kernel": _BUILD_N30_S9},
     "vggt_n800_s9": {"global_attn_kernel": _ATTN_N30_S9 * 800 / 30, "build_kv_kernel": _BUILD_N30_S9 * 800 / 30},
@@ -299,7 +299,14 @@ def run_ours(args, wl):
     dev = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
-    shard_mode = world > 1 and not args.replicas
+    elif args.shard:
+        # the frame-sharded path with a group of one rank (no peer, same calls): a check of that path on one GPU
+        import socket
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+        dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1, device_id=dev)
+    shard_mode = (world > 1 and not args.replicas) or (world == 1 and args.shard)
     stream = torch.cuda.current_stream(dev)
     H, d = wl.n_heads, wl.head_dim
 
@@ -520,6 +527,7 @@ def run_ours(args, wl):
         print(json.dumps(line))
     if world > 1:
         dist.barrier()
+    if dist.is_initialized():
         dist.destroy_process_group()
 
 
@@ -534,6 +542,8 @@ def main():
     ap.add_argument("--no-dense", action="store_true", help="skip the dense (s = 1) comparison run")
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-configuration report")
     ap.add_argument("--no-projection", action="store_true", help="skip the fused projection + compaction timing")
+    ap.add_argument("--shard", action="store_true",
+                    help="with one GPU: run the frame-sharded path with a one-rank group (checks that path; not the default)")
     ap.add_argument("--replicas", action="store_true",
                     help="with N > 1: N independent copies of the problem instead of one problem split by frames")
     args = ap.parse_args()
