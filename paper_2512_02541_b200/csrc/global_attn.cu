@@ -26,10 +26,10 @@
 // Tensor memory per tile: S 128 columns (fp32), P 64 columns (bf16 pairs),
 // O 64 columns (fp32); 512 columns in all.  A softmax thread pulls its 64 scores
 // of S into registers and the warp frees its rows at once, so the next Q K^T runs
-// under the exponentials; P V of step j runs under the softmax of step j+1.  The
-// two tiles take turns in the exponential phase.  The accumulator is rescaled
-// lazily: only when the running maximum grew by more than 2^8 since the last
-// rescale.  The epilogue folds the diagonal and the mean-fill column into the
+// under the exponentials; P V of step j runs under the softmax of step j+1.  One
+// pair of scores in eight takes its exponential from a polynomial on the FMA
+// pipe.  The accumulator is rescaled lazily: only when the running maximum grew
+// by more than 2^8 since the last rescale.  The epilogue folds the diagonal and the mean-fill column into the
 // same normalisation:
 //   O = (a_S O_S + p_d v_i + p_m vmean) / (a_S l_S + p_d + p_m).
 #include <mutex>
@@ -50,7 +50,10 @@ constexpr int kQTiles = 2;       // tiles per CTA
 constexpr int kTileKV = 128;     // keys per step
 constexpr int kHeadDim = 64;
 constexpr uint32_t kTileBytes = kTileKV * kHeadDim * 2;   // 16 KiB: one 128 x 64 bf16 tile
-constexpr int kStages = 3;       // K ring and V ring depth
+#ifndef AVGGT_STAGES
+#define AVGGT_STAGES 3
+#endif
+constexpr int kStages = AVGGT_STAGES;       // K ring and V ring depth
 constexpr int kThreads = 640;
 constexpr int kSoftmaxWarps = 16;
 constexpr int kTmaWarp = 16;
@@ -61,23 +64,11 @@ constexpr uint32_t kColP = 128, kColO = 192;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 
-// Of every 8 pairs of scores, this many take their exponential from a polynomial on the FMA
-// pipe instead of the special-function unit (which, at 16 results per clock per SM, is the
-// scarcest resource of the softmax at head dimension 64).
+// Of every 8 pairs of scores, this many take their exponential from a polynomial on the FMA pipe instead of the
+// special-function unit (which, at 16 results per clock per SM, is the scarcest arithmetic unit of the softmax at
+// head dimension 64).  One in eight measured best: 754 ms against 784 ms on the 800-frame layer; two in eight 768 ms.
 #ifndef AVGGT_POLY_EIGHTHS
-#define AVGGT_POLY_EIGHTHS 0
-#endif
-// 1: the softmax warps of the two query tiles that share a scheduler take turns in the
-// exponential phase (two warps at a time saturate the unit), so that one tile's waits, loads,
-// maxima and stores run under the other tile's exponentials instead of all four warps
-// marching in step.
-#ifndef AVGGT_PINGPONG
-#define AVGGT_PINGPONG 1
-#endif
-// The turn is handed to the other tile after this group of 32 keys (0..3) of a step; 3 = at the end.  Handing over
-// early lets the other tile's warps wake up and start while this tile still feeds the exponential unit.
-#ifndef AVGGT_HANDOVER_GROUP
-#define AVGGT_HANDOVER_GROUP 1
+#define AVGGT_POLY_EIGHTHS 1
 #endif
 constexpr int kPolyEighths = AVGGT_POLY_EIGHTHS;
 
@@ -111,7 +102,6 @@ struct __align__(8) Barriers {
   uint64_t s_free[kQTiles];    // softmax -> MMA: S_t(j) has been read into registers
   uint64_t p_full[kQTiles];    // softmax -> MMA: P_t(j) stored (and O_t rescaled)
   uint64_t o_done[kQTiles];    // MMA -> softmax: P_t(j) V_j has completed
-  uint64_t turn[kQTiles][4];   // both warps of rows [32 q, 32 q + 32) of the other tile -> this tile's: the exponential unit is yours
   uint64_t mma_idle[kQTiles];  // MMA issuer t -> itself: every tcgen05.mma it issued has completed
   uint32_t tmem_base;
   uint32_t abort_flag;
@@ -422,9 +412,10 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1
   p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
 }
 
-// pair g (0..7 within a group of eight) goes to the polynomial when kPoly of eight do
+// Block b of 8 key columns (0..15 within a step) goes to the polynomial when kPoly of eight blocks do.  The choice
+// depends on the column alone, so a query row's result does not depend on where in a tile the row sits.
 template <int kPoly>
-__device__ __forceinline__ constexpr bool pair_uses_poly(int g) { return ((g + 1) * kPoly) / 8 != (g * kPoly) / 8; }
+__device__ __forceinline__ constexpr bool block_uses_poly(int b) { return (((b & 7) + 1) * kPoly) / 8 != ((b & 7) * kPoly) / 8; }
 
 // What a softmax thread knows about itself.  A softmax warp works on 16 query rows of its tile, all 128 columns
 // of a key step: the tensor-memory lanes [32 q + 16 h, 32 q + 16 h + 16) of the tile.  Its tensor-memory
@@ -515,8 +506,7 @@ struct RowState {
 // pair in dependency order; the instruction scheduler interleaves the pairs.
 template <bool kLse, int kPoly>
 __device__ __forceinline__ void softmax_rows(const uint32_t (&s)[64], uint64_t scale2, const uint64_t (&neg_m2)[2],
-                                             float (&sum_lo)[2], float (&sum_hi)[2], uint64_t (&sum_exact2)[2], uint32_t tP,
-                                             uint32_t turn_bar, int lane) {
+                                             float (&sum_lo)[2], float (&sum_hi)[2], uint64_t (&sum_exact2)[2], uint32_t tP) {
 #pragma unroll
   for (int g = 0; g < 4; ++g) {
     uint32_t pk[8];   // P of 32 keys x 2 rows as bf16 pairs
@@ -527,7 +517,7 @@ __device__ __forceinline__ void softmax_rows(const uint32_t (&s)[64], uint64_t s
         const int c = 4 * (4 * g + n) + 2 * hi;
         const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), scale2, neg_m2[hi]);
         float p0, p1;
-        if (pair_uses_poly<kPoly>(2 * n + hi)) {
+        if (block_uses_poly<kPoly>(4 * g + n)) {
           exp2_poly_pair(x2, p0, p1);
         } else {
           float x0, x1;
@@ -542,13 +532,6 @@ __device__ __forceinline__ void softmax_rows(const uint32_t (&s)[64], uint64_t s
       }
     }
     tmem_st_rows16_p16(tP + g * 16, pk);
-#if AVGGT_PINGPONG
-    // the store above is ordered before the arrival, and with it this group's exponentials
-    if (g == AVGGT_HANDOVER_GROUP) {
-      __syncwarp();
-      if (lane == 0) mbar_arrive(turn_bar);
-    }
-#endif
   }
 }
 
@@ -558,8 +541,8 @@ __device__ __forceinline__ void softmax_rows(const uint32_t (&s)[64], uint64_t s
 // The 64 scores are pulled into registers at once and the warp's share of S_t is released, so that the next
 // Q K^T runs under this step's exponentials.  The row maxima (two shuffles within the quad) decide whether a
 // reference maximum moves (lazy rescale).
-// j: step within the work item; g: the tile's steps in the CTA's earlier work items.  kPoly: pairs per eight
-// whose exponential is a polynomial.  kLse: also keep the sum of the unrounded exponentials, for the
+// j: step within the work item; g: the tile's steps in the CTA's earlier work items.  kPoly: blocks of 8 columns per eight
+// whose exponentials are polynomials.  kLse: also keep the sum of the unrounded exponentials, for the
 // log-sum-exp output.  kMasked: columns >= valid are excluded (valid may be <= 0).
 template <bool kMasked, bool kLse, int kPoly>
 __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int g, int valid, float scale_log2,
@@ -611,10 +594,6 @@ __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int
     for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha[(c >> 1) & 1]);
     tmem_st_rows16_c64(me.tO, o);
   }
-#if AVGGT_PINGPONG
-  // this tile's turn on the exponential unit: the other tile's two warps on this scheduler have left their phase
-  if (!wait_bar(&bars->turn[me.t][me.q], gj & 1, bars, a, 62 + me.t, gj)) return false;
-#endif
 
   // exponentials, rounded to bf16 for the value product; the normaliser sums the
   // rounded values so that numerator and denominator carry the same weights
@@ -622,8 +601,7 @@ __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int
   const uint64_t neg_m2[2] = {pack_f32x2(-st.m_used[0], -st.m_used[0]), pack_f32x2(-st.m_used[1], -st.m_used[1])};
   float sum_lo[2] = {0.f, 0.f}, sum_hi[2] = {0.f, 0.f};   // even and odd columns
   uint64_t sum_exact2[2] = {pack_f32x2(0.f, 0.f), pack_f32x2(0.f, 0.f)};
-  softmax_rows<kLse, kPoly>(s, scale2, neg_m2, sum_lo, sum_hi, sum_exact2, me.tP,
-                            smem_u32(&bars->turn[me.t ^ 1][me.q]), me.lane);
+  softmax_rows<kLse, kPoly>(s, scale2, neg_m2, sum_lo, sum_hi, sum_exact2, me.tP);
 #pragma unroll
   for (int hi = 0; hi < 2; ++hi) {
     st.l_run[hi] += sum_lo[hi] + sum_hi[hi];
@@ -794,10 +772,6 @@ __device__ __forceinline__ void softmax_role(const AttnArgs& a, Barriers* bars, 
   me.tS = tile_base;
   me.tP = tile_base + kColP;
   me.tO = tile_base + kColO;
-#if AVGGT_PINGPONG
-  // tile 0 goes first: tile 1 hands it the first turn
-  if (me.t == 1 && lane == 0) mbar_arrive(smem_u32(&bars->turn[0][me.q]));
-#endif
   const int n_kv = a.n_kv_tiles;
   int g = 0, n_done = 0;
 #pragma unroll 1
@@ -840,7 +814,6 @@ global_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       mbar_init(smem_u32(&bars.s_free[t]), kSoftmaxWarps / kQTiles);
       mbar_init(smem_u32(&bars.p_full[t]), kSoftmaxWarps / kQTiles);
       mbar_init(smem_u32(&bars.o_done[t]), 1);
-      for (int w = 0; w < 4; ++w) mbar_init(smem_u32(&bars.turn[t][w]), 2);
       mbar_init(smem_u32(&bars.mma_idle[t]), 1);
       mbar_init(smem_u32(&bars.o_free[t]), kSoftmaxWarps / kQTiles);
     }
