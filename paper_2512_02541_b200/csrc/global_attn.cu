@@ -50,10 +50,12 @@ constexpr int kQTiles = 2;       // tiles per CTA
 constexpr int kTileKV = 128;     // keys per step
 constexpr int kHeadDim = 64;
 constexpr uint32_t kTileBytes = kTileKV * kHeadDim * 2;   // 16 KiB: one 128 x 64 bf16 tile
+// K ring and V ring depth.  The subsampled layer runs the same at 2 to 5; frame attention, whose strided key
+// tiles take longer to arrive, gained 6 % from the fourth stage and nothing from a fifth.
 #ifndef AVGGT_STAGES
-#define AVGGT_STAGES 3
+#define AVGGT_STAGES 4
 #endif
-constexpr int kStages = AVGGT_STAGES;       // K ring and V ring depth
+constexpr int kStages = AVGGT_STAGES;
 constexpr int kThreads = 640;
 constexpr int kSoftmaxWarps = 16;
 constexpr int kTmaWarp = 16;
@@ -493,6 +495,21 @@ __device__ __forceinline__ float quad_sum(float v) {
   return v + __shfl_xor_sync(0xffffffffu, v, 2);
 }
 
+// 4 x 4 transpose over a quad: thread i gives word b and ends with the four words that the threads 0..3 held in
+// their place i (two exchanges, with the neighbour at distance 1 and then 2; every lane of the warp takes part)
+__device__ __forceinline__ void quad_transpose(uint32_t& w0, uint32_t& w1, uint32_t& w2, uint32_t& w3, int i) {
+  const bool odd = (i & 1) != 0, upper = (i & 2) != 0;
+  uint32_t got;
+  got = __shfl_xor_sync(0xffffffffu, odd ? w0 : w1, 1);
+  if (odd) w0 = got; else w1 = got;
+  got = __shfl_xor_sync(0xffffffffu, odd ? w2 : w3, 1);
+  if (odd) w2 = got; else w3 = got;
+  got = __shfl_xor_sync(0xffffffffu, upper ? w0 : w2, 2);
+  if (upper) w0 = got; else w2 = got;
+  got = __shfl_xor_sync(0xffffffffu, upper ? w1 : w3, 2);
+  if (upper) w1 = got; else w3 = got;
+}
+
 // Running state of the thread's two rows (the same in all four threads of a quad, except the partial sums).
 struct RowState {
   float m_used[2];    // reference maximum of the stored exponentials (log2 units)
@@ -504,14 +521,21 @@ struct RowState {
 // probabilities, stored to tensor memory at tP, relative to the rows' reference maxima folded into neg_m2; adds
 // to the sums for the normaliser (of the rounded values) and for the log-sum-exp (unrounded).  Written pair by
 // pair in dependency order; the instruction scheduler interleaves the pairs.
-template <bool kLse, int kPoly>
+template <bool kMasked, bool kLse, int kPoly>
 __device__ __forceinline__ void softmax_rows(const uint32_t (&s)[64], uint64_t scale2, const uint64_t (&neg_m2)[2],
-                                             float (&sum_lo)[2], float (&sum_hi)[2], uint64_t (&sum_exact2)[2], uint32_t tP) {
+                                             float (&sum_lo)[2], float (&sum_hi)[2], uint64_t (&sum_exact2)[2], uint32_t tP,
+                                             int n_blocks) {
 #pragma unroll
   for (int g = 0; g < 4; ++g) {
     uint32_t pk[8];   // P of 32 keys x 2 rows as bf16 pairs
 #pragma unroll
     for (int n = 0; n < 4; ++n) {
+      // ragged last step: a block of 8 columns with no key in it gives zeros without any arithmetic
+      if (kMasked && 4 * g + n >= n_blocks) {
+        pk[2 * n] = 0u;
+        pk[2 * n + 1] = 0u;
+        continue;
+      }
 #pragma unroll
       for (int hi = 0; hi < 2; ++hi) {
         const int c = 4 * (4 * g + n) + 2 * hi;
@@ -601,7 +625,8 @@ __device__ __forceinline__ bool softmax_step(const SoftmaxThread& me, int j, int
   const uint64_t neg_m2[2] = {pack_f32x2(-st.m_used[0], -st.m_used[0]), pack_f32x2(-st.m_used[1], -st.m_used[1])};
   float sum_lo[2] = {0.f, 0.f}, sum_hi[2] = {0.f, 0.f};   // even and odd columns
   uint64_t sum_exact2[2] = {pack_f32x2(0.f, 0.f), pack_f32x2(0.f, 0.f)};
-  softmax_rows<kLse, kPoly>(s, scale2, neg_m2, sum_lo, sum_hi, sum_exact2, me.tP);
+  const int n_blocks = kMasked ? (valid + 7) >> 3 : 16;   // blocks of 8 columns that hold a key
+  softmax_rows<kMasked, kLse, kPoly>(s, scale2, neg_m2, sum_lo, sum_hi, sum_exact2, me.tP, n_blocks);
 #pragma unroll
   for (int hi = 0; hi < 2; ++hi) {
     st.l_run[hi] += sum_lo[hi] + sum_hi[hi];
@@ -642,7 +667,8 @@ __device__ __forceinline__ bool softmax_item(const AttnArgs& a, Barriers* bars, 
     const int valid = static_cast<int>(a.n_keys - static_cast<int64_t>(j) * kTileKV);
     bool ok;
     // the masked (last, ragged) tile keeps every exponential on the special-function unit, where -inf gives an exact 0
-    if (valid < kTileKV) ok = softmax_step<true, true, 0>(me, j, g, valid, a.scale_log2, st, bars, a);
+    if (valid < kTileKV) ok = want_lse ? softmax_step<true, true, 0>(me, j, g, valid, a.scale_log2, st, bars, a)
+                                       : softmax_step<true, false, 0>(me, j, g, valid, a.scale_log2, st, bars, a);
     else if (want_lse) ok = softmax_step<false, true, kPolyEighths>(me, j, g, valid, a.scale_log2, st, bars, a);
     else ok = softmax_step<false, false, kPolyEighths>(me, j, g, valid, a.scale_log2, st, bars, a);
     if (!ok) return false;
@@ -685,14 +711,14 @@ __device__ __forceinline__ bool softmax_item(const AttnArgs& a, Barriers* bars, 
     const int r = me.r[hi];
     const int row = cta.q0 + t * kTileQ + r;           // query token
     const bool row_valid = row < cta.row_end;
-    bool is_dropped = false;
-    if (row_valid && pl.n_dropped > 0) {
+    bool is_dropped = false;   // only the diagonal term asks
+    if (a.use_diag && row_valid) {
       const int32_t f = row / pl.L;
       is_dropped = (a.slot_of_token != nullptr ? a.slot_of_token[row] : compact_slot(pl, f, row - f * pl.L)) < 0;
     }
     // the row's sums over its four threads
     const float l_run = quad_sum(st.l_run[hi]);
-    const float l_exact = quad_sum(st.l_exact[hi]);
+    const float l_exact = want_lse ? quad_sum(st.l_exact[hi]) : 0.f;
     const float m_used = st.m_used[hi];
     // base-2 logits of the two extra columns: each thread of the quad takes its 16 dimensions, then the quad adds up
     // (every thread runs the shuffles; rows without the term carry zeros)
@@ -719,36 +745,48 @@ __device__ __forceinline__ bool softmax_item(const AttnArgs& a, Barriers* bars, 
       acc_d = quad_sum(acc_d);
       acc_m = quad_sum(acc_m);
     }
-    float l_d = -INFINITY, l_m = -INFINITY;
-    if (has_diag) l_d = acc_d * a.scale_log2;
-    if (has_mean) {
-      l_m = acc_m * a.scale_log2;
-      if (pl.mean_fill == AVGGT_MEAN_FILL) l_m += log2f(static_cast<float>(count));
-    }
-    const float m_fin = fmaxf(m_used, fmaxf(l_d, l_m));
-    const float a_s = exp2f(m_used - m_fin);
-    const float p_d = exp2f(l_d - m_fin);              // 0 when the term is absent
-    const float p_m = exp2f(l_m - m_fin);
-    const float z = fmaf(l_run, a_s, p_d + p_m);
-    const float inv_z = 1.0f / z;
-    const float w_s = a_s * inv_z, w_d = p_d * inv_z, w_m = p_m * inv_z;
-    if (row_valid) {
-      uint32_t* dst = reinterpret_cast<uint32_t*>(a.O + (static_cast<size_t>(row) * pl.H + head) * kHeadDim);
-#pragma unroll
-      for (int b = 0; b < 8; ++b) {
-        float v0 = __uint_as_float(o[4 * b + 2 * hi]) * w_s, v1 = __uint_as_float(o[4 * b + 2 * hi + 1]) * w_s;
-        if (w_d != 0.f) {
-          const uint32_t vw = ld_swizzled_word(sVd, r, 4 * b + me.i);
-          v0 = fmaf(w_d, __uint_as_float(vw << 16), v0);
-          v1 = fmaf(w_d, __uint_as_float(vw & 0xffff0000u), v1);
-        }
-        if (has_mean) {
-          const float2 vm = __ldg(reinterpret_cast<const float2*>(a.vmean + head * kHeadDim + 8 * b + 2 * me.i));
-          v0 = fmaf(w_m, vm.x, v0);
-          v1 = fmaf(w_m, vm.y, v1);
-        }
-        dst[4 * b + me.i] = pack_bf16x2(v0, v1);
+    float m_fin = m_used, a_s = 1.0f, p_d = 0.f, p_m = 0.f;
+    if (a.use_diag || a.use_mean) {   // the same for every row of the launch; frame attention has neither
+      float l_d = -INFINITY, l_m = -INFINITY;
+      if (has_diag) l_d = acc_d * a.scale_log2;
+      if (has_mean) {
+        l_m = acc_m * a.scale_log2;
+        if (pl.mean_fill == AVGGT_MEAN_FILL) l_m += log2f(static_cast<float>(count));
       }
+      m_fin = fmaxf(m_used, fmaxf(l_d, l_m));
+      a_s = exp2f(m_used - m_fin);
+      p_d = exp2f(l_d - m_fin);              // 0 when the term is absent
+      p_m = exp2f(l_m - m_fin);
+    }
+    const float z = fmaf(l_run, a_s, p_d + p_m);
+    const float inv_z = __fdividef(1.0f, z);   // z is at least one exponential of a row maximum, far from the ends of the range
+    const float w_s = a_s * inv_z, w_d = p_d * inv_z, w_m = p_m * inv_z;
+    // the thread's 8 words of the output row: word 4 b + i (dimensions 8 b + 2 i, 8 b + 2 i + 1)
+    uint32_t w[8];
+#pragma unroll
+    for (int b = 0; b < 8; ++b) {
+      float v0 = __uint_as_float(o[4 * b + 2 * hi]) * w_s, v1 = __uint_as_float(o[4 * b + 2 * hi + 1]) * w_s;
+      if (w_d != 0.f) {
+        const uint32_t vw = ld_swizzled_word(sVd, r, 4 * b + me.i);
+        v0 = fmaf(w_d, __uint_as_float(vw << 16), v0);
+        v1 = fmaf(w_d, __uint_as_float(vw & 0xffff0000u), v1);
+      }
+      if (has_mean) {
+        const float2 vm = __ldg(reinterpret_cast<const float2*>(a.vmean + head * kHeadDim + 8 * b + 2 * me.i));
+        v0 = fmaf(w_m, vm.x, v0);
+        v1 = fmaf(w_m, vm.y, v1);
+      }
+      w[b] = pack_bf16x2(v0, v1);
+    }
+    // Transposed within the quad, a thread holds 16 contiguous bytes of each half of the row: 4 stores of 16 bytes
+    // per thread instead of 16 of 4 bytes (whose 8 rows x 16 bytes per warp instruction kept the store path of the
+    // SM busy for thousands of clocks per work item).
+    quad_transpose(w[0], w[1], w[2], w[3], me.i);
+    quad_transpose(w[4], w[5], w[6], w[7], me.i);
+    if (row_valid) {
+      uint4* dst = reinterpret_cast<uint4*>(a.O + (static_cast<size_t>(row) * pl.H + head) * kHeadDim);
+      dst[me.i] = make_uint4(w[0], w[1], w[2], w[3]);
+      dst[4 + me.i] = make_uint4(w[4], w[5], w[6], w[7]);
       if (want_lse && me.i == 0) {
         const float z_exact = fmaf(l_exact, a_s, p_d + p_m);
         a.lse[static_cast<size_t>(row) * pl.H + head] = (m_fin + log2f(z_exact)) * 0.6931471805599453f;
