@@ -42,7 +42,7 @@ from paper_2512_02541_b200 import inputs  # noqa: E402
 # profiles/; None where no capture covers the workload.  Both kernels are captured on the 30-frame copy of the
 # headline layer (profiles/*_vggt_n30_s9.md); their traffic is proportional to the frame count, so the 800-frame
 # figures are those captures x 800/30.
-_ATTN_N30_S9 = 0.275052544e9 + 0.066984192e9
+_ATTN_N30_S9 = 0.275011072e9 + 0.067811584e9
 _BUILD_N30_S9 = 0.168855296e9 + 0.009879808e9
 NCU_TRAFFIC = {
     "vggt_n30_s9": {"global_attn_kernel": _ATTN_N30_S9, "build_kv_kernel": _BUILD_N30_S9},
