@@ -138,21 +138,6 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Barrier
   }
 }
 
-// 16-byte chunk c (0..7) of row r of a 128-byte-swizzled tile
-__device__ __forceinline__ uint4 ld_swizzled(const uint8_t* tile, int r, int c) {
-  return *reinterpret_cast<const uint4*>(tile + r * 128 + ((c ^ (r & 7)) << 4));
-}
-
-__device__ __forceinline__ float dot_bf16x8(const uint4& a, const uint4& b, float acc) {
-  const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    acc = fmaf(__uint_as_float(aw[i] << 16), __uint_as_float(bw[i] << 16), acc);
-    acc = fmaf(__uint_as_float(aw[i] & 0xffff0000u), __uint_as_float(bw[i] & 0xffff0000u), acc);
-  }
-  return acc;
-}
-
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));

@@ -12,7 +12,12 @@
 //   warp 1      MMA issuer: tcgen05.mma, M 128 x N 256 x K 16, fp32 accumulators in tensor memory;
 //               two accumulators of 256 columns, so the next tile's products run under this
 //               tile's epilogue
-//   warps 2-5   epilogue, one token row per thread: accumulator -> registers, bias, bf16, stores;
+//   warps 2-9   epilogue, one token row and half of the tile's columns per thread: accumulator -> registers, bias, bf16; a head's
+//               64 values of the warp's 32 rows are staged in shared memory (128-byte swizzle),
+//               from where one TMA store writes them to the full K / V array and the retained
+//               rows are copied, 128 contiguous bytes at a time, to the compact arrays (a thread
+//               storing its own row 16 bytes at a time kept the store path busy for longer than
+//               the products of the tile take);
 //               the sums over dropped rows are taken across the 32 rows of a warp with a
 //               transposing shuffle reduction (lane c ends up with column c) and kept in
 //               registers for all the tiles of the CTA
@@ -38,7 +43,10 @@ constexpr int kBlockK = 64;       // channels per ring stage: one 128-byte swizz
 constexpr int kProjStages = 4;
 constexpr uint32_t kBytesA = kTileTok * kBlockK * 2;   // 16 KiB
 constexpr uint32_t kBytesB = kTileCol * kBlockK * 2;   // 32 KiB
-constexpr int kProjThreads = 192;   // warps 2..5 are the epilogue: warp % 4 covers the four lane quarters of tensor memory
+constexpr uint32_t kStageBytes = 32 * 128;   // epilogue staging: 32 rows x one head (64 bf16), one per epilogue warp
+constexpr int kEpiWarps = 8;        // warps 2..9: warp % 4 is the lane quarter of tensor memory, (warp - 2) / 4 the half of
+                                    // the tile's 256 columns (two heads each)
+constexpr int kProjThreads = 64 + 32 * kEpiWarps;
 constexpr uint32_t kProjTmemCols = 512;
 
 struct ProjArgs {
@@ -117,11 +125,13 @@ __device__ __forceinline__ float warp_column_sums(float (&v)[32], int lane) {
 
 __global__ void __launch_bounds__(kProjThreads, 1)
 project_kv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_wk,
-                  const __grid_constant__ CUtensorMap tm_wv, const ProjArgs a) {
+                  const __grid_constant__ CUtensorMap tm_wv, const __grid_constant__ CUtensorMap tm_kfull,
+                  const __grid_constant__ CUtensorMap tm_vfull, const ProjArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sA = smem;                               // kProjStages tiles of X
   uint8_t* sB = smem + kProjStages * kBytesA;       // kProjStages tiles of W
+  uint8_t* sStage = sB + kProjStages * kBytesB;     // one staging tile per epilogue warp
   __shared__ ProjBarriers bars;
 
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0);
@@ -142,7 +152,7 @@ project_kv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&bars.acc_full[b]), 1);
-      mbar_init(smem_u32(&bars.acc_empty[b]), 4);
+      mbar_init(smem_u32(&bars.acc_empty[b]), kEpiWarps);
     }
     mbar_init(smem_u32(&bars.mma_idle), 1);
     bars.abort_flag = 0;
@@ -226,13 +236,16 @@ project_kv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     // ------------------------------------------------------------ epilogue: one token row per thread
     const Plan& pl = a.pl;
     const int quarter = warp & 3;                       // tensor-memory lanes [32 quarter, 32 quarter + 32)
+    const int col_half = (warp - 2) >> 2;               // columns [128 col_half, 128 col_half + 128) of the tile
+    uint8_t* sbuf = sStage + (warp - 2) * kStageBytes;
     const float* bias = which == 0 ? a.bias_k : a.bias_v;
-    uint4* full = which == 0 ? a.K_full : a.V_full;
+    const bool write_full = (which == 0 ? a.K_full : a.V_full) != nullptr;
+    const CUtensorMap* tm_full = which == 0 ? &tm_kfull : &tm_vfull;
     uint4* compact = which == 0 ? a.Kc : a.Vc;
     const int cols_total = pl.H * pl.d;
-    float colsum[kTileCol / 32];                        // lane c: column 32 i + c of this CTA's block, over dropped rows
+    float colsum[4];                                    // lane c: column 128 col_half + 32 i + c of this CTA's block, over dropped rows
 #pragma unroll
-    for (int i = 0; i < kTileCol / 32; ++i) colsum[i] = 0.f;
+    for (int i = 0; i < 4; ++i) colsum[i] = 0.f;
     int it = 0;
     bool ok = true;
     for (int tt = tok0; tt < a.n_tok_tiles; tt += a.tok_stride, ++it) {
@@ -240,48 +253,74 @@ project_kv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       ok = proj_wait_warp(&bars.acc_full[buf], (it >> 1) & 1, &bars, a, 30, it);
       if (!ok) break;
       tc_fence_after();
-      const int64_t row = static_cast<int64_t>(tt) * kTileTok + quarter * 32 + lane;
+      const int64_t row0 = static_cast<int64_t>(tt) * kTileTok + quarter * 32;   // first row of this warp
+      const int64_t row = row0 + lane;
       const bool row_valid = row < pl.n_tok;
       int32_t cs = -1;
-      int64_t m = 0;
+      int32_t m = 0;
       if (row_valid) {
         const int32_t f = static_cast<int32_t>(row / pl.L);
         cs = compact_slot(pl, f, static_cast<int32_t>(row - static_cast<int64_t>(f) * pl.L));
-        if (cs >= 0) m = compact_frame_base(pl, f) + cs;
+        if (cs >= 0) m = static_cast<int32_t>(compact_frame_base(pl, f) + cs);
       }
       const bool kept = row_valid && cs >= 0;
       const bool dropped = row_valid && cs < 0;
-      if (kept && which == 0 && col_tile == 0 && a.idx != nullptr) a.idx[m] = static_cast<int32_t>(row);
+      if (kept && which == 0 && col_tile == 0 && col_half == 0 && a.idx != nullptr) a.idx[m] = static_cast<int32_t>(row);
+      const uint32_t kept_mask = __ballot_sync(0xffffffffu, kept);
+      const int n_kept = __popc(kept_mask);
       const uint32_t t_acc = tmem + buf * kTileCol + (static_cast<uint32_t>(32 * quarter) << 16);
 #pragma unroll
-      for (int c = 0; c < kTileCol / 32; ++c) {
-        uint32_t raw[32];
-        tmem_ld32(t_acc + c * 32, raw);
-        tmem_wait_ld();
-        const int col0 = col_tile * kTileCol + c * 32;            // first column of the chunk within K (or V)
-        if (col0 < cols_total) {                                    // warp-uniform: a chunk is half a head
+      for (int hh = 0; hh < 2; ++hh) {                              // one head (64 columns) at a time
+        const int hg = 2 * col_half + hh;                           // head within the tile
+        const int col0 = col_tile * kTileCol + hg * 64;             // first column within K (or V)
+        if (col0 >= cols_total) break;                              // warp-uniform: H * d is a multiple of 64
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t raw[32];
+          tmem_ld32(t_acc + hg * 64 + half * 32, raw);
+          tmem_wait_ld();
           float v[32];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(raw[i]) + (bias != nullptr ? __ldg(bias + col0 + i) : 0.f);
-          uint4 out[4];
-          uint32_t* o32 = reinterpret_cast<uint32_t*>(out);
-#pragma unroll
-          for (int i = 0; i < 16; ++i) o32[i] = pack_bf16x2(v[2 * i], v[2 * i + 1]);
-          const int head = col0 >> 6, dchunk = (col0 & 63) >> 3;    // 16-byte chunk within the head's 64 values
-          if (row_valid && full != nullptr) {
-            uint4* dst = full + (static_cast<size_t>(row) * pl.H + head) * 8 + dchunk;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) dst[i] = out[i];
+          for (int i = 0; i < 32; ++i)
+            v[i] = __uint_as_float(raw[i]) + (bias != nullptr ? __ldg(bias + col0 + half * 32 + i) : 0.f);
+          if (half == 0) {
+            // the store of the previous head has finished reading the staging tile
+            if (lane == 0) bulk_wait_read<0>();
+            __syncwarp();
           }
-          if (kept) {
-            uint4* dst = compact + (static_cast<size_t>(head) * static_cast<size_t>(pl.M) + static_cast<size_t>(m)) * 8 + dchunk;
+          // row `lane` of the staging tile, 16-byte chunks 4 half .. 4 half + 3, swizzled as TMA expects them
 #pragma unroll
-            for (int i = 0; i < 4; ++i) dst[i] = out[i];
+          for (int i = 0; i < 4; ++i) {
+            uint4 o;
+            o.x = pack_bf16x2(v[8 * i], v[8 * i + 1]);
+            o.y = pack_bf16x2(v[8 * i + 2], v[8 * i + 3]);
+            o.z = pack_bf16x2(v[8 * i + 4], v[8 * i + 5]);
+            o.w = pack_bf16x2(v[8 * i + 6], v[8 * i + 7]);
+            *reinterpret_cast<uint4*>(sbuf + lane * 128 + (((4 * half + i) ^ (lane & 7)) << 4)) = o;
           }
           if (a.do_mean) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = dropped ? v[i] : 0.f;
-            colsum[c] += warp_column_sums(v, lane);
+            colsum[2 * hh + half] += warp_column_sums(v, lane);
+          }
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        // every row of the tile to the full array (rows beyond the last token are clipped by the tensor map)
+        if (write_full && lane == 0) {
+          tma_store_2d(tm_full, smem_u32(sbuf), col0, static_cast<int>(row0));
+          bulk_commit();
+        }
+        // retained rows to the compact array: four rows per pass, eight lanes x 16 bytes per row
+        const int head = col0 >> 6;
+        for (int k0 = 0; k0 < n_kept; k0 += 4) {
+          const int k = k0 + (lane >> 3);
+          const bool have = k < n_kept;
+          const int r = have ? static_cast<int>(__fns(kept_mask, 0, k + 1)) : 0;
+          const int32_t m_r = __shfl_sync(0xffffffffu, m, r);
+          if (have) {
+            const uint4 val = *reinterpret_cast<const uint4*>(sbuf + r * 128 + (((lane & 7) ^ (r & 7)) << 4));
+            compact[(static_cast<size_t>(head) * static_cast<size_t>(pl.M) + static_cast<size_t>(m_r)) * 8 + (lane & 7)] = val;
           }
         }
       }
@@ -290,10 +329,12 @@ project_kv_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars.acc_empty[buf]));
     }
+    if (lane == 0) bulk_wait<0>();   // the staging tiles stay put until the last store has read them
+    __syncwarp();
     if (ok && a.do_mean) {
-      float* dst = a.partials + (static_cast<size_t>(blockIdx.x) * 4 + quarter) * kTileCol;
+      float* dst = a.partials + (static_cast<size_t>(blockIdx.x) * 4 + quarter) * kTileCol + 128 * col_half;
 #pragma unroll
-      for (int i = 0; i < kTileCol / 32; ++i) dst[32 * i + lane] = colsum[i];
+      for (int i = 0; i < 4; ++i) dst[32 * i + lane] = colsum[i];
     }
   }
 
@@ -317,7 +358,7 @@ project_mean_kernel(const float* __restrict__ partials, int grid, int n_col_tile
   (which == 0 ? kmean : vmean)[col] = s * inv_count;
 }
 
-constexpr size_t kProjSmemBytes = static_cast<size_t>(kProjStages) * (kBytesA + kBytesB) + 1024;
+constexpr size_t kProjSmemBytes = static_cast<size_t>(kProjStages) * (kBytesA + kBytesB) + 8 * kStageBytes + 1024;
 
 int project_grid(const Plan& pl, int sm_count) {
   const int per_tok = 2 * ((pl.H * pl.d + kTileCol - 1) / kTileCol);
@@ -357,7 +398,7 @@ cudaError_t launch_project_kv(const Plan& pl, int sm_count, int model_dim, const
   a.partials = reinterpret_cast<float*>(static_cast<char*>(ws) + kAttnStatusBytes);
   a.do_mean = (pl.mean_fill != 0 && pl.n_dropped > 0) ? 1 : 0;
 
-  CUtensorMap tm_x, tm_wk, tm_wv;
+  CUtensorMap tm_x, tm_wk, tm_wv, tm_kfull, tm_vfull;
   const uint64_t x_dims[2] = {static_cast<uint64_t>(model_dim), static_cast<uint64_t>(pl.n_tok)};
   const uint64_t w_dims[2] = {static_cast<uint64_t>(model_dim), static_cast<uint64_t>(cols_total)};
   const uint64_t row_bytes[1] = {static_cast<uint64_t>(model_dim) * 2};
@@ -366,13 +407,22 @@ cudaError_t launch_project_kv(const Plan& pl, int sm_count, int model_dim, const
   bool good = make_tmap_bf16(&tm_x, X, 2, x_dims, row_bytes, x_box);
   good = good && make_tmap_bf16(&tm_wk, Wk, 2, w_dims, row_bytes, w_box);
   good = good && make_tmap_bf16(&tm_wv, Wv, 2, w_dims, row_bytes, w_box);
+  // the full K / V arrays as [n_tok, H * d], written 32 rows x one head at a time (any valid map stands in for an
+  // array that is not wanted; the kernel does not use it then)
+  const uint64_t f_dims[2] = {static_cast<uint64_t>(cols_total), static_cast<uint64_t>(pl.n_tok)};
+  const uint64_t f_row_bytes[1] = {static_cast<uint64_t>(cols_total) * 2};
+  const uint32_t f_box[2] = {64, 32};
+  if (K != nullptr) good = good && make_tmap_bf16(&tm_kfull, K, 2, f_dims, f_row_bytes, f_box);
+  else tm_kfull = tm_x;
+  if (V != nullptr) good = good && make_tmap_bf16(&tm_vfull, V, 2, f_dims, f_row_bytes, f_box);
+  else tm_vfull = tm_x;
   if (!good) { *tmap_failed = true; return cudaSuccess; }
 
   cudaError_t e = cudaFuncSetAttribute(project_kv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kProjSmemBytes));
   if (e != cudaSuccess) return e;
   e = cudaMemsetAsync(ws, 0, kAttnStatusBytes, st);
   if (e != cudaSuccess) return e;
-  project_kv_kernel<<<grid, kProjThreads, kProjSmemBytes, st>>>(tm_x, tm_wk, tm_wv, a);
+  project_kv_kernel<<<grid, kProjThreads, kProjSmemBytes, st>>>(tm_x, tm_wk, tm_wv, tm_kfull, tm_vfull, a);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (pl.mean_fill != 0) {
