@@ -69,30 +69,43 @@ class SubsampledGlobalAttention:
         K and V go to the device first (the compaction and the mean need all of them); Q then arrives in
         ``n_chunks`` groups of frames on a copy stream while the attention of the previous group runs
         (``avggt_global_attn_shard``: the queries of a frame range against the whole sequence's compact keys), and
-        every group's output leaves on a second copy stream.  Everything is ordered with events; on return the
-        current stream waits for the last output copy.  The device staging buffers are allocated on first use.
+        every group's output leaves on a second copy stream.  Everything is ordered with events and the call
+        returns without waiting for the device: the current stream waits for the last output copy.  The device
+        copies of K and V alternate between two buffers, so that the K and V of a call made right after this one
+        travel while this one's attention runs; Q and O have one buffer, guarded group by group.  The device
+        staging buffers are allocated on first use.
         """
         p = self.params
         dev = self.device
         cur = torch.cuda.current_stream(dev)
         if not hasattr(self, "_host_path"):
             shape = (self.n_tok, p.n_heads, p.head_dim)
+            new = lambda: torch.empty(shape, dtype=torch.bfloat16, device=dev)
             self._host_path = dict(
-                Q=torch.empty(shape, dtype=torch.bfloat16, device=dev), K=torch.empty(shape, dtype=torch.bfloat16, device=dev),
-                V=torch.empty(shape, dtype=torch.bfloat16, device=dev), O=torch.empty(shape, dtype=torch.bfloat16, device=dev),
-                h2d=torch.cuda.Stream(dev), d2h=torch.cuda.Stream(dev),
+                Q=new(), O=new(), K=[new(), new()], V=[new(), new()], h2d=torch.cuda.Stream(dev), d2h=torch.cuda.Stream(dev),
+                calls=0,
+                kv_free=[None, None],    # per K/V buffer: the call that used it last has finished with it
+                bounds=None,             # frame groups of the previous call
+                q_free=[], o_free=[],    # per group of the previous call: its attention has read Q / its output copy has left O
                 # one status block per group of frames, so that no launch clears what an earlier one reported
                 ws=torch.zeros((max(1, p.n_frames), max(self.attn_ws_bytes, 256)), dtype=torch.uint8, device=dev))
         hp = self._host_path
-        dQ, dK, dV, dO, h2d, d2h = hp["Q"], hp["K"], hp["V"], hp["O"], hp["h2d"], hp["d2h"]
+        which = hp["calls"] & 1
+        hp["calls"] += 1
+        dQ, dK, dV, dO, h2d, d2h = hp["Q"], hp["K"][which], hp["V"][which], hp["O"], hp["h2d"], hp["d2h"]
         L = p.tokens_per_frame
         n_chunks = max(1, min(n_chunks, p.n_frames))
         bounds = [round(i * p.n_frames / n_chunks) for i in range(n_chunks + 1)]
+        same_groups = hp["bounds"] == bounds
         keep_first = bool(p.flags & B.AVGGT_FLAG_KEEP_FIRST_FRAME)
-        h2d.wait_stream(cur)
-        d2h.wait_stream(cur)
+        if not same_groups:
+            # the previous call cut the frames differently: wait for all of it before Q and O are touched
+            h2d.wait_stream(cur)
+            h2d.wait_stream(d2h)
         with torch.cuda.device(dev):
             with torch.cuda.stream(h2d):
+                if hp["kv_free"][which] is not None:
+                    h2d.wait_event(hp["kv_free"][which])
                 dK.copy_(hK, non_blocking=True)
                 dV.copy_(hV, non_blocking=True)
                 kv_ready = torch.cuda.Event()
@@ -100,12 +113,15 @@ class SubsampledGlobalAttention:
                 q_ready = []
                 for c in range(n_chunks):
                     sl = slice(bounds[c] * L, bounds[c + 1] * L)
+                    if same_groups:
+                        h2d.wait_event(hp["q_free"][c])
                     dQ[sl].copy_(hQ[sl], non_blocking=True)
                     ev = torch.cuda.Event()
                     ev.record(h2d)
                     q_ready.append(ev)
             cur.wait_event(kv_ready)
             self.build_kv(dK, dV)
+            q_free, o_free = [], []
             for c in range(n_chunks):
                 f0, f1 = bounds[c], bounds[c + 1]
                 sl = slice(f0 * L, f1 * L)
@@ -113,13 +129,21 @@ class SubsampledGlobalAttention:
                                    mean_fill=p.mean_fill, softmax_scale=p.softmax_scale,
                                    keep_first_frame=keep_first and f0 == 0)
                 cur.wait_event(q_ready[c])
+                if same_groups:
+                    cur.wait_event(hp["o_free"][c])
                 B.avggt_global_attn_shard(cp, self.M, self.n_dropped, dQ[sl], dK[sl], dV[sl], self.Kc, self.Vc, self.kmean,
                                           self.vmean, dO[sl], None, hp["ws"][c], hp["ws"][c].numel(), cur.cuda_stream)
                 done = torch.cuda.Event()
                 done.record(cur)
+                q_free.append(done)
                 d2h.wait_event(done)
                 with torch.cuda.stream(d2h):
                     hO[sl].copy_(dO[sl], non_blocking=True)
+                    left = torch.cuda.Event()
+                    left.record(d2h)
+                    o_free.append(left)
+            hp["kv_free"][which] = q_free[-1]
+            hp["bounds"], hp["q_free"], hp["o_free"] = bounds, q_free, o_free
             cur.wait_stream(d2h)
         return hO
 

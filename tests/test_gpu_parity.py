@@ -292,7 +292,7 @@ def test_extreme_values_stay_finite():
 def test_host_buffer_forward_matches_the_device_forward():
     """forward_host (K/V first, Q in groups of frames on a copy stream, outputs leaving on another) gives the very
     bits of forward on resident tensors, for a frame count that does not divide into the groups, with and without
-    the uncompressed first frame."""
+    the uncompressed first frame; also for calls that follow one another without a wait."""
     for kff in (0, 1):
         wl = inputs.Workload("host", 11, 12, 13, 5, 4, 64, 4, 1, 2, "proj", keep_first_frame=kff)
         params, ocfg = _cfgs(wl)
@@ -307,3 +307,15 @@ def test_host_buffer_forward_matches_the_device_forward():
             layer.forward_host(hQ, hK, hV, hO, n_chunks=n_chunks)
             layer.check_status()
             assert torch.equal(hO, O.cpu()), n_chunks
+        # three calls in a row without waiting in between, on two different inputs: the K and V of a call travel
+        # (to the other of the two device buffers) while the attention of the call before runs
+        Q2, K2, V2 = inputs.make_qkv(wl, seed=22, device="cuda")
+        O2 = layer.forward(Q2, K2, V2).clone()
+        layer.check_status()
+        hQ2, hK2, hV2 = (t.cpu().pin_memory() for t in (Q2, K2, V2))
+        outs = [torch.full_like(hQ, float("nan")).pin_memory() for _ in range(3)]
+        layer.forward_host(hQ, hK, hV, outs[0], n_chunks=4)
+        layer.forward_host(hQ2, hK2, hV2, outs[1], n_chunks=4)
+        layer.forward_host(hQ, hK, hV, outs[2], n_chunks=4)
+        layer.check_status()
+        assert torch.equal(outs[0], O.cpu()) and torch.equal(outs[1], O2.cpu()) and torch.equal(outs[2], O.cpu())
