@@ -231,6 +231,25 @@ def _layer_for(P, wl, dev, sigma=None, diag=None, mean_fill=None):
     return P.SubsampledGlobalAttention(params, device=dev)
 
 
+def input_logit_stats(wl, Q, K, n=1024):
+    """What the synthetic inputs look like to the softmax (harness arithmetic, head 0, patch queries of frame 1):
+    scaled logits of a query against its own key, against the key at the same grid position of frame 0 (the
+    cross-view correspondence the input recipe plants) and against random other keys."""
+    if wl.n_frames < 2 or wl.grid_h * wl.grid_w < 1:
+        return None
+    L = wl.tokens_per_frame
+    g = torch.Generator(device=Q.device).manual_seed(7)
+    slots = wl.n_special + torch.randint(0, wl.grid_h * wl.grid_w, (n,), generator=g, device=Q.device)
+    rows = L + slots
+    q = Q[rows, 0].float()
+    scale = wl.head_dim ** -0.5
+    own = (q * K[rows, 0].float()).sum(-1) * scale
+    same = (q * K[slots, 0].float()).sum(-1) * scale
+    other = (q * K[torch.randint(0, wl.n_tokens, (n,), generator=g, device=Q.device), 0].float()).sum(-1) * scale
+    return {"own_key_mean": float(own.mean()), "same_position_other_frame_mean": float(same.mean()),
+            "other_keys_mean": float(other.mean()), "other_keys_std": float(other.std()), "sampled_queries": n}
+
+
 def time_config(P, wl, Q, K, V, O, dev, peaks, launches=3):
     """A few launches of the whole path on one configuration (inputs resident): per-kernel times from CUDA events."""
     stream = torch.cuda.current_stream(dev)
@@ -327,6 +346,7 @@ def run_ours(args, wl):
         units_all = world * wl.n_tokens
         n_q_local = wl.n_tokens
     O = torch.empty_like(Q)
+    logits = input_logit_stats(wl, Q, K) if (rank == 0 and not shard_mode) else None
 
     def barrier():
         if world > 1:
@@ -493,7 +513,7 @@ def run_ours(args, wl):
             "config": {"workload": wl.name, "n_frames": wl.n_frames, "grid": [wl.grid_h, wl.grid_w],
                        "n_special": wl.n_special, "heads": H, "head_dim": d, "sigma": wl.sigma, "diag": wl.diag,
                        "mean_fill": wl.mean_fill, "queries": wl.n_tokens, "compact_keys": M,
-                       "l2": "inputs_larger_than_l2", "parallelism": par},
+                       "l2": "inputs_larger_than_l2", "parallelism": par, "input_logits": logits},
             "tflops": 4.0 * units_all * M * H * d / (ms_per_step * 1e-3) / 1e12,
             "attn_ms": attn_avg, "attn_ms_min": min(attn_ms), "build_kv_ms": build_avg, "build_kv_ms_min": min(build_ms),
             "exchange_ms": exch_avg if shard_mode else None,
