@@ -27,10 +27,10 @@
 // O 64 columns (fp32); 512 columns in all.  A softmax thread pulls its 64 scores
 // of S into registers and the warp frees its rows at once, so the next Q K^T runs
 // under the exponentials; P V of step j runs under the softmax of step j+1.  One
-// pair of scores in eight takes its exponential from a polynomial on the FMA
-// pipe.  The accumulator is rescaled lazily: only when the running maximum grew
-// by more than 2^8 since the last rescale.  The epilogue folds the diagonal and the mean-fill column into the
-// same normalisation:
+// block of 8 key columns in eight takes its exponentials from a polynomial on
+// the FMA pipe.  The accumulator is rescaled lazily: only when the running
+// maximum grew by more than 2^8 since the last rescale.  The epilogue folds the
+// diagonal and the mean-fill column into the same normalisation:
 //   O = (a_S O_S + p_d v_i + p_m vmean) / (a_S l_S + p_d + p_m).
 #include <mutex>
 
@@ -66,9 +66,10 @@ constexpr uint32_t kColP = 128, kColO = 192;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 
-// Of every 8 pairs of scores, this many take their exponential from a polynomial on the FMA pipe instead of the
-// special-function unit (which, at 16 results per clock per SM, is the scarcest arithmetic unit of the softmax at
-// head dimension 64).  One in eight measured best: 754 ms against 784 ms on the 800-frame layer; two in eight 768 ms.
+// Of every 8 blocks of 8 key columns, this many take their exponentials from a polynomial on the FMA pipe instead of
+// the special-function unit (which, at 16 results per clock per SM, is the scarcest arithmetic unit of the softmax at
+// head dimension 64).  One in eight measured best: 723 ms on the 800-frame layer against 768 ms with none and 767 ms
+// with two in eight.
 #ifndef AVGGT_POLY_EIGHTHS
 #define AVGGT_POLY_EIGHTHS 1
 #endif
