@@ -26,7 +26,7 @@
  *     AVGGT_ERR_CUDA, the clearing of the status block may already be on the
  *     stream; no kernel is.)  No exception crosses this boundary.
  *   - Size limits: head_dim == 64; n_heads <= 32; batch == 1;
- *     N * L <= 2^31 - 257 tokens; frame attention: N <= 65535 frames.  Anything
+ *     N * L <= 2^31 - 257 tokens; frame attention: ceil(L / 256) * H * N < 2^31.  Anything
  *     beyond them is rejected with AVGGT_ERR_UNSUPPORTED.
  *   - Only sm_100 devices are supported (AVGGT_ERR_UNSUPPORTED elsewhere).
  *     There is no CPU fallback.
@@ -300,7 +300,7 @@ int avggt_shard_assemble(const avggt_params* p, const void* gathered, int32_t n_
  * N independent dense problems in one launch of the same kernel; keys and values are read
  * straight from K and V (nothing is compacted), so avggt_build_kv is not needed.  Of `p` the
  * call uses n_frames, tokens_per_frame, n_heads, head_dim and softmax_scale; sigma, diag,
- * mean_fill and flags play no part but must be valid.  n_frames <= 65535.
+ * mean_fill and flags play no part but must be valid.  ceil(L / 256) * H * N < 2^31.
  *
  *   Q, K, V       device, bf16 [N*L, H, d]; must be finite (a tile of keys may reach into the
  *                 next frame's rows, whose products are masked to zero weight)

@@ -334,7 +334,8 @@ int avggt_frame_attn(const avggt_params* p, const void* Q, const void* K, const 
   Plan pl;
   int rc = make_plan(p, &pl);
   if (rc != AVGGT_OK) return rc;
-  if (pl.n_frames > 65535) return AVGGT_ERR_UNSUPPORTED;
+  // one work item per pair of 128-row query tiles, head and frame; their number is a 32-bit count in the kernel
+  if ((static_cast<int64_t>(pl.L) + 255) / 256 * pl.H * pl.n_frames > 2147483647LL) return AVGGT_ERR_UNSUPPORTED;
   return run_attn(pl, AttnCall{Q, K, V, nullptr, nullptr, nullptr, nullptr, O, lse, ws, ws_bytes, cuda_stream, nullptr, true});
 }
 

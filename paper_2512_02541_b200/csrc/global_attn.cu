@@ -84,7 +84,7 @@ struct AttnArgs {
   const int32_t* slot_of_token;   // caller-chosen retained set: compact position of every token, -1 = dropped; else null
   uint32_t* status;     // 4 words
   int32_t frame_mode;   // 0: subsampled global attention over the compact keys.  1: frame attention (Sec. 4.2):
-                        //    blockIdx.z is the frame, keys and values are the frame's own rows of K and V
+                        //    every frame is a problem of its own, keys and values are the frame's own rows of K and V
   int64_t n_keys;       // keys of one problem: M, or the tokens of a frame
   int32_t n_kv_tiles;   // ceil(n_keys / 128)
   int32_t n_work;       // work items (pairs of query tiles x heads x problems) of the launch; a CTA takes the items

@@ -75,6 +75,14 @@ def test_argument_validation_codes():
     assert b"unknown" in binding.lib().avggt_strerror(-99)
 
 
+def test_frame_attention_work_item_limit_is_checked_on_the_host():
+    """ceil(L / 256) * H * N work items must fit a 32-bit count: rejected before any device call."""
+    p = P.make_params(1 << 26, 1, 1, 1, 32, 64, 4)     # 2 tokens per frame, 2^27 tokens, 2^31 work items
+    lib = binding.lib()
+    assert lib.avggt_kv_count(ctypes.byref(p), None, None) == 0
+    assert lib.avggt_frame_attn(ctypes.byref(p), None, None, None, None, None, None, 0, None) == -2
+
+
 def test_product_does_not_import_the_oracle():
     pkg = os.path.join(ROOT, "paper_2512_02541_b200")
     for dirpath, _, files in os.walk(pkg):
